@@ -1,0 +1,163 @@
+/*
+ * wush.h - C ABI of the B200 (sm_100a) W4A4 WUSH linear-layer library.
+ *
+ * Method: "WUSH: Near-Optimal Adaptive Transforms for LLM Quantization"
+ * (arXiv 2512.00956).  The online layer (Eq. 7, Sec. 5 "GPU Kernel Support") is
+ *
+ *     Y = sum_i  W~_(i)^T  q( T_wush(i)  X~_(i) )
+ *
+ * with block-diagonal transforms of block size d = g, q the round-to-nearest AbsMax
+ * block quantiser over groups of g consecutive input channels (Sec. 3, "Block-
+ * independent constraint"), and W~_(i) = q(T_xvsh(i) W_(i)) prepared offline
+ * (Algorithm 2, RTN case) with T_xvsh = T_wush^-T (Eq. 6).
+ *
+ * Layout bridge.  The paper writes column vectors (X in R^{d_in x d_batch}, output
+ * W^T X).  This library is row-major:  X[M,K], W[N,K], Y[M,N] = X W^T, with
+ * M = d_batch, K = d_in, N = d_out, g = d, C = K/g.  T_(i) x on a column block is
+ *     v[m, c*g + j] = sum_k T[c][j][k] * x[m, c*g + k].
+ *
+ * Formats.  MXFP4: g = 32, E2M1 codes, one E8M0 scale byte per block
+ * (2^(byte-127), byte = 127 + floor(log2 AbsMax) - 2, clamped to [0,254]).
+ * NVFP4: g = 16, E2M1 codes, one E4M3 scale byte per block and one fp32 scale per
+ * tensor; with a = AbsMax of the block the scale byte is E4M3(round-nearest-even,
+ * saturate 448) of (a / 6) / tensor_scale, elements are multiplied by
+ * 1 / (float(scale byte) * tensor_scale) and rounded to E2M1 (nearest, ties to the
+ * even code, saturate at 6, sign kept).  Two codes per byte, element 2t in the low
+ * nibble.  NaN/Inf inputs are not detected (they saturate).
+ *
+ * Conventions for every entry point
+ *   - all data pointers are DEVICE pointers owned by the caller unless a parameter is
+ *     documented as "host"; the library does not allocate, free or retain them;
+ *   - work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and the call returns without synchronising;
+ *   - the return value is a wush_status_t: 0 on success, negative on error.
+ *     Argument errors are found on the host before anything is launched, and then
+ *     no output is touched.
+ *   - base pointers must be 16-byte aligned; K must be a multiple of 64.
+ */
+#ifndef WUSH_H_
+#define WUSH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  WUSH_OK = 0,
+  WUSH_ERR_NULL = -1,      /* a required pointer is NULL */
+  WUSH_ERR_SHAPE = -2,     /* non-positive size, K % g != 0, K % 64 != 0, N % 8 != 0 ... */
+  WUSH_ERR_FORMAT = -3,    /* unknown format / layout, or g does not match the format */
+  WUSH_ERR_ALIGN = -4,     /* a base pointer is not 16-byte aligned */
+  WUSH_ERR_WORKSPACE = -5, /* workspace missing or smaller than wush_*_workspace_bytes() */
+  WUSH_ERR_CUDA = -6,      /* a CUDA call or launch failed; see wush_last_cuda_error() */
+  WUSH_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (reported by wush_gemm_status) */
+  WUSH_ERR_DEVICE = -8     /* the current device is not compute capability 10.x */
+} wush_status_t;
+
+typedef enum { WUSH_MXFP4 = 0, WUSH_NVFP4 = 1 } wush_format_t;
+
+/* Scale-byte layouts.
+ *  LINEAR: scales[row][K/g], row-major.
+ *  TILED : the layout the block-scaled tensor-core GEMM consumes.  Rows are padded to a
+ *          multiple of 128 and scale columns to a multiple of 4; the byte of (row r,
+ *          scale column kb) lives at
+ *              ((r/128) * ceil(K/g/4) + kb/4) * 512 + (r%32)*16 + ((r%128)/32)*4 + kb%4.
+ *          Padding bytes are never read for valid outputs and are left untouched.
+ *          Size: wush_scale_bytes(rows, K, g, WUSH_SF_TILED). */
+typedef enum { WUSH_SF_LINEAR = 0, WUSH_SF_TILED = 1 } wush_sf_layout_t;
+
+typedef enum { WUSH_OUT_F32 = 0, WUSH_OUT_BF16 = 1 } wush_out_t;
+
+const char* wush_status_string(int status);
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char* wush_last_cuda_error(void);
+
+/* Bytes of a scale buffer for `rows` rows in the given layout (0 on bad arguments). */
+size_t wush_scale_bytes(int64_t rows, int64_t K, int g, wush_sf_layout_t sf);
+
+/* ---------------------------------------------------------------------------------------
+ * Online step 1 (Eq. 7 inner term, Sec. 5 "Fused WUSH + Quant kernel"):
+ *   codes, scales = q( X_blk * T_c^T )  for every token row and every block c.
+ *   X      bf16 [M,K] row-major.
+ *   T      bf16 [K/g][g][g]; T[c][j][k] multiplies input channel c*g+k into output
+ *          coordinate c*g+j (the activation-side transform T_wush of Eq. 5, stored as
+ *          16-bit values, Sec. 3 "Costs for online inference").
+ *   x_tensor_scale  fp32[1] on the device; NVFP4 only (static, chosen at calibration
+ *          time), must be > 0; pass NULL for MXFP4.
+ *   codes  uint8 [M, K/2];  scales uint8, layout `sf`.
+ * Errors: NULL / SHAPE / FORMAT / ALIGN / CUDA.  M = 0 is a no-op returning WUSH_OK. */
+int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T,
+                      wush_format_t fmt, int g, const float* x_tensor_scale,
+                      uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf, void* stream);
+
+/* Offline weight preparation (Algorithm 2, RTN case, last line):
+ *   W~ = q( W_blk * Tinv_c^T ),  Tinv = T_xvsh = T_wush^-T (Eq. 6) given in fp32.
+ *   W      bf16 [N,K];  Tinv fp32 [K/g][g][g] (same index convention as T above).
+ *   w_tensor_scale  fp32[1] on the device, WRITTEN for NVFP4: AbsMax of the whole
+ *          transformed tensor / (6*448); ignored (may be NULL) for MXFP4.
+ *   workspace       device scratch of at least wush_quantize_weight_workspace_bytes();
+ *          contents on entry are irrelevant; must not be shared by overlapping calls.
+ * The product is evaluated on tensor cores from an exact 3-way bf16 split of Tinv with
+ * fp32 accumulation.  Errors as above plus WORKSPACE. */
+int wush_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv,
+                         wush_format_t fmt, int g, float* w_tensor_scale,
+                         uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf,
+                         void* workspace, size_t workspace_bytes, void* stream);
+size_t wush_quantize_weight_workspace_bytes(int64_t N, int64_t K, wush_format_t fmt, int g);
+
+/* Online step 2 (Eq. 7 outer sum): block-scaled FP4 GEMM on tcgen05 tensor cores,
+ *   Y[m,n] = alpha * sum_c sx[m,c] * sw[n,c] * sum_{k in c} xq[m,k] * wq[n,k],
+ *   alpha = 1 (MXFP4) or x_tensor_scale * w_tensor_scale (NVFP4), fp32 accumulation.
+ *   Xq [M,K/2], Wq [N,K/2] packed codes; Xs, Ws scale bytes in TILED layout.
+ *   Y  [M,N] row-major, fp32 or bf16 (`ydt`).  N must be a multiple of 8.
+ *   status  optional int32[1] on the device: set to a non-zero diagnostic word if a
+ *           bounded wait inside the kernel expired (then Y is undefined); may be NULL.
+ * Errors: NULL / SHAPE / FORMAT / ALIGN / DEVICE / CUDA. */
+int wush_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws,
+                  int64_t M, int64_t N, int64_t K, wush_format_t fmt, int g,
+                  const float* x_tensor_scale, const float* w_tensor_scale,
+                  void* Y, wush_out_t ydt, int32_t* status, void* stream);
+
+/* The whole online layer (Eq. 7): wush_quantize_act into `workspace`, then wush_gemm_fp4,
+ * both on `stream`.  Wcodes/Wscales come from wush_quantize_weight with WUSH_SF_TILED.
+ * workspace: at least wush_linear_workspace_bytes(M, K, g) bytes, 16-byte aligned.  Its
+ * last 16 bytes receive the GEMM's status word (see wush_gemm_fp4). */
+int wush_linear(const void* X, int64_t M, int64_t K, const void* T,
+                const uint8_t* Wcodes, const uint8_t* Wscales, int64_t N,
+                const float* x_tensor_scale, const float* w_tensor_scale,
+                wush_format_t fmt, int g, void* Y, wush_out_t ydt,
+                void* workspace, size_t workspace_bytes, void* stream);
+size_t wush_linear_workspace_bytes(int64_t M, int64_t K, int g);
+
+/* Offline calibration statistics (Algorithm 2, first line of the RTN loop):
+ *   moments[c] += sum_t  x_{t,c}^T x_{t,c}   (unnormalised g x g second moment of block c)
+ *   *count     += B
+ *   Xc       bf16 [B,K] (calibration activations, or the weight matrix W[N,K] itself
+ *            for the weight-side moment);  moments fp32 [K/g][g][g], accumulated in
+ *            place so calibration can be fed in chunks; count int64[1] on the device.
+ *   workspace device scratch of at least wush_calib_moments_workspace_bytes(B,K,g).
+ * The reduction order is fixed, so results are run-to-run identical. */
+int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* moments,
+                       int64_t* count, void* workspace, size_t workspace_bytes, void* stream);
+size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g);
+
+/* ----------------------------------------------------------------- diagnostic exports */
+/* The block quantiser q(.) alone on fp32 input V[R,K] (same outputs as above). */
+int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, int g,
+                      const float* tensor_scale, uint8_t* codes, uint8_t* scales,
+                      wush_sf_layout_t sf, void* stream);
+/* The block transform alone: V[M,K] fp32 = X_blk * T_c^T, same arithmetic as
+ * wush_quantize_act uses before quantising. */
+int wush_transform_act_f32(const void* X, int64_t M, int64_t K, const void* T, int g,
+                           float* V, void* stream);
+/* Same for the weight side (fp32 Tinv, 3-way split). */
+int wush_transform_weight_f32(const void* W, int64_t N, int64_t K, const float* Tinv, int g,
+                              float* V, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WUSH_H_ */

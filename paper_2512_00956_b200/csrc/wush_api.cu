@@ -1,0 +1,208 @@
+// extern "C" entry points of libwush: argument validation and dispatch.  See include/wush.h
+// for the contract of every call.
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/wush.h"
+#include "wush_device.cuh"
+#include "wush_host.h"
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char* why = nullptr) {
+  snprintf(g_cuda_error, sizeof(g_cuda_error), "%s%s%s", cudaGetErrorString(e), why ? ": " : "", why ? why : "");
+  return WUSH_ERR_CUDA;
+}
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int check_fmt(int fmt, int g) {
+  if (fmt == WUSH_MXFP4) return g == 32 ? WUSH_OK : WUSH_ERR_FORMAT;
+  if (fmt == WUSH_NVFP4) return g == 16 ? WUSH_OK : WUSH_ERR_FORMAT;
+  return WUSH_ERR_FORMAT;
+}
+inline int check_shape(int64_t rows, int64_t K, int g) {
+  if (rows < 0 || K <= 0 || g <= 0) return WUSH_ERR_SHAPE;
+  if (K % g != 0 || K % 64 != 0) return WUSH_ERR_SHAPE;
+  if (rows > (int64_t)1 << 30 || K > (int64_t)1 << 30) return WUSH_ERR_SHAPE;
+  return WUSH_OK;
+}
+inline size_t round16(size_t x) { return (x + 15) & ~size_t(15); }
+
+bool device_is_sm100() {
+  static int cached = -1;
+  if (cached < 0) {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
+    cached = (major == 10) ? 1 : 0;
+  }
+  return cached == 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* wush_status_string(int status) {
+  switch (status) {
+    case WUSH_OK: return "ok";
+    case WUSH_ERR_NULL: return "null pointer";
+    case WUSH_ERR_SHAPE: return "bad shape";
+    case WUSH_ERR_FORMAT: return "bad format / group size / layout";
+    case WUSH_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case WUSH_ERR_WORKSPACE: return "workspace missing or too small";
+    case WUSH_ERR_CUDA: return "CUDA error";
+    case WUSH_ERR_TIMEOUT: return "bounded device wait expired";
+    case WUSH_ERR_DEVICE: return "device is not compute capability 10.x";
+    default: return "unknown status";
+  }
+}
+
+const char* wush_last_cuda_error(void) { return g_cuda_error; }
+
+size_t wush_scale_bytes(int64_t rows, int64_t K, int g, wush_sf_layout_t sf) {
+  if (rows < 0 || K <= 0 || (g != 16 && g != 32) || K % g != 0) return 0;
+  const int64_t KB = K / g;
+  if (sf == WUSH_SF_LINEAR) return (size_t)(rows * KB);
+  if (sf == WUSH_SF_TILED) return (size_t)(((rows + 127) / 128) * ((KB + 3) / 4) * 512);
+  return 0;
+}
+
+int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T, wush_format_t fmt, int g,
+                      const float* x_tensor_scale, uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf,
+                      void* stream) {
+  int rc = check_fmt(fmt, g);
+  if (rc) return rc;
+  if ((rc = check_shape(M, K, g))) return rc;
+  if (sf != WUSH_SF_LINEAR && sf != WUSH_SF_TILED) return WUSH_ERR_FORMAT;
+  if (!X || !T || !codes || !scales || (fmt == WUSH_NVFP4 && !x_tensor_scale)) return WUSH_ERR_NULL;
+  if (!aligned16(X) || !aligned16(T) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
+  if (M == 0) return WUSH_OK;
+  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+size_t wush_quantize_weight_workspace_bytes(int64_t, int64_t, wush_format_t, int) { return 256; }
+
+int wush_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv, wush_format_t fmt, int g,
+                         float* w_tensor_scale, uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_fmt(fmt, g);
+  if (rc) return rc;
+  if ((rc = check_shape(N, K, g))) return rc;
+  if (sf != WUSH_SF_LINEAR && sf != WUSH_SF_TILED) return WUSH_ERR_FORMAT;
+  if (!W || !Tinv || !codes || !scales || (fmt == WUSH_NVFP4 && !w_tensor_scale)) return WUSH_ERR_NULL;
+  if (!workspace || workspace_bytes < wush_quantize_weight_workspace_bytes(N, K, fmt, g)) return WUSH_ERR_WORKSPACE;
+  if (!aligned16(W) || !aligned16(Tinv) || !aligned16(codes) || !aligned16(scales) || !aligned16(workspace))
+    return WUSH_ERR_ALIGN;
+  if (N == 0) return WUSH_OK;
+  cudaError_t e = wush::run_quantize_weight(W, N, K, Tinv, g, w_tensor_scale, codes, scales, (int)sf,
+                                            reinterpret_cast<uint32_t*>(workspace), (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+int wush_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws, int64_t M,
+                  int64_t N, int64_t K, wush_format_t fmt, int g, const float* x_tensor_scale,
+                  const float* w_tensor_scale, void* Y, wush_out_t ydt, int32_t* status, void* stream) {
+  int rc = check_fmt(fmt, g);
+  if (rc) return rc;
+  if ((rc = check_shape(M, K, g))) return rc;
+  if (N <= 0 || N % 8 != 0 || N > (int64_t)1 << 30) return WUSH_ERR_SHAPE;
+  if (ydt != WUSH_OUT_F32 && ydt != WUSH_OUT_BF16) return WUSH_ERR_FORMAT;
+  if (!Xq || !Xs || !Wq || !Ws || !Y) return WUSH_ERR_NULL;
+  if (fmt == WUSH_NVFP4 && (!x_tensor_scale || !w_tensor_scale)) return WUSH_ERR_NULL;
+  if (!aligned16(Xq) || !aligned16(Xs) || !aligned16(Wq) || !aligned16(Ws) || !aligned16(Y)) return WUSH_ERR_ALIGN;
+  if (M == 0) return WUSH_OK;
+  if (!device_is_sm100()) return WUSH_ERR_DEVICE;
+  const char* why = nullptr;
+  cudaError_t e = wush::run_gemm_fp4(Xq, Xs, Wq, Ws, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
+                                     ydt == WUSH_OUT_BF16, status, (cudaStream_t)stream, &why);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e, why);
+}
+
+size_t wush_linear_workspace_bytes(int64_t M, int64_t K, int g) {
+  if (M < 0 || K <= 0 || (g != 16 && g != 32) || K % g != 0) return 0;
+  return round16((size_t)(M * (K / 2))) + round16(wush_scale_bytes(M, K, g, WUSH_SF_TILED)) + 16;
+}
+
+int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_t* Wcodes,
+                const uint8_t* Wscales, int64_t N, const float* x_tensor_scale, const float* w_tensor_scale,
+                wush_format_t fmt, int g, void* Y, wush_out_t ydt, void* workspace, size_t workspace_bytes,
+                void* stream) {
+  int rc = check_fmt(fmt, g);
+  if (rc) return rc;
+  if ((rc = check_shape(M, K, g))) return rc;
+  if (!workspace || workspace_bytes < wush_linear_workspace_bytes(M, K, g)) return WUSH_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return WUSH_ERR_ALIGN;
+  uint8_t* xq = reinterpret_cast<uint8_t*>(workspace);
+  uint8_t* xs = xq + round16((size_t)(M * (K / 2)));
+  int32_t* status = reinterpret_cast<int32_t*>(xs + round16(wush_scale_bytes(M, K, g, WUSH_SF_TILED)));
+  // validate the GEMM's arguments before the quantiser touches anything
+  if (N <= 0 || N % 8 != 0) return WUSH_ERR_SHAPE;
+  if (ydt != WUSH_OUT_F32 && ydt != WUSH_OUT_BF16) return WUSH_ERR_FORMAT;
+  if (!X || !T || !Wcodes || !Wscales || !Y) return WUSH_ERR_NULL;
+  if (fmt == WUSH_NVFP4 && (!x_tensor_scale || !w_tensor_scale)) return WUSH_ERR_NULL;
+  if (!aligned16(Wcodes) || !aligned16(Wscales) || !aligned16(Y)) return WUSH_ERR_ALIGN;
+  rc = wush_quantize_act(X, M, K, T, fmt, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, stream);
+  if (rc) return rc;
+  return wush_gemm_fp4(xq, xs, Wcodes, Wscales, M, N, K, fmt, g, x_tensor_scale, w_tensor_scale, Y, ydt, status,
+                       stream);
+}
+
+size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g) {
+  if (B < 0 || K <= 0 || (g != 16 && g != 32) || K % g != 0) return 0;
+  return (size_t)wush::moments_splits(B, K) * (size_t)K * (size_t)g * sizeof(float);
+}
+
+int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* moments, int64_t* count,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+  if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  int rc = check_shape(B, K, g);
+  if (rc) return rc;
+  if (!Xc || !moments || !count) return WUSH_ERR_NULL;
+  if (!workspace || workspace_bytes < wush_calib_moments_workspace_bytes(B, K, g)) return WUSH_ERR_WORKSPACE;
+  if (!aligned16(Xc) || !aligned16(moments) || !aligned16(workspace)) return WUSH_ERR_ALIGN;
+  if (B == 0) return WUSH_OK;
+  cudaError_t e = wush::run_calib_moments(Xc, B, K, g, moments, count, reinterpret_cast<float*>(workspace),
+                                          wush::moments_splits(B, K), (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, int g, const float* tensor_scale,
+                      uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf, void* stream) {
+  int rc = check_fmt(fmt, g);
+  if (rc) return rc;
+  if ((rc = check_shape(R, K, g))) return rc;
+  if (sf != WUSH_SF_LINEAR && sf != WUSH_SF_TILED) return WUSH_ERR_FORMAT;
+  if (!V || !codes || !scales || (fmt == WUSH_NVFP4 && !tensor_scale)) return WUSH_ERR_NULL;
+  if (!aligned16(V) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
+  if (R == 0) return WUSH_OK;
+  cudaError_t e = wush::run_quantize_f32(V, R, K, g, tensor_scale, codes, scales, (int)sf, (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+int wush_transform_act_f32(const void* X, int64_t M, int64_t K, const void* T, int g, float* V, void* stream) {
+  if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  int rc = check_shape(M, K, g);
+  if (rc) return rc;
+  if (!X || !T || !V) return WUSH_ERR_NULL;
+  if (!aligned16(X) || !aligned16(T) || !aligned16(V)) return WUSH_ERR_ALIGN;
+  if (M == 0) return WUSH_OK;
+  cudaError_t e = wush::run_transform_f32(X, M, K, T, g, false, V, (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+int wush_transform_weight_f32(const void* W, int64_t N, int64_t K, const float* Tinv, int g, float* V,
+                              void* stream) {
+  if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  int rc = check_shape(N, K, g);
+  if (rc) return rc;
+  if (!W || !Tinv || !V) return WUSH_ERR_NULL;
+  if (!aligned16(W) || !aligned16(Tinv) || !aligned16(V)) return WUSH_ERR_ALIGN;
+  if (N == 0) return WUSH_OK;
+  cudaError_t e = wush::run_transform_f32(W, N, K, Tinv, g, true, V, (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+}  // extern "C"

@@ -1,0 +1,87 @@
+// Device-side helpers shared by the kernels of libwush: scale-layout indexing, the
+// E2M1 / E8M0 / E4M3 block quantiser q(.) of Sec. 3 ("Block-independent constraint"),
+// and the warp-level bf16 tensor-core instruction used for the g x g block products.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp4.h>
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace wush {
+
+constexpr int kFmtMX = 0;   // MXFP4: g = 32, E8M0 scale
+constexpr int kFmtNV = 1;   // NVFP4: g = 16, E4M3 scale + fp32 tensor scale
+
+// Byte offset of the scale of (row r, scale column kb) in a buffer with KB scale columns.
+// layout 0: [rows][KB];  layout 1: 128-row x 4-column tiles of 512 bytes, the order the
+// block-scaled MMA reads from tensor memory (32 lanes x 16 bytes, four 32-row groups
+// interleaved at 4-byte granularity).
+__host__ __device__ __forceinline__ int64_t sf_offset(int layout, int64_t r, int64_t kb, int64_t KB) {
+  if (layout == 0) return r * KB + kb;
+  const int64_t ktiles = (KB + 3) >> 2;
+  return ((r >> 7) * ktiles + (kb >> 2)) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4 + (kb & 3);
+}
+
+// ---- E2M1: round to nearest (ties to the even code), saturate at 6, keep the sign.
+// Packs 8 fp32 values into 8 nibbles, element 0 in the lowest nibble.
+__device__ __forceinline__ uint32_t pack_e2m1x8(const float (&u)[8]) {
+  uint32_t w = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_fp4x2_storage_t b =
+        __nv_cvt_float2_to_fp4x2(make_float2(u[2 * i], u[2 * i + 1]), __NV_E2M1, cudaRoundNearest);
+    w |= static_cast<uint32_t>(b) << (8 * i);
+  }
+  return w;
+}
+
+// ---- MXFP4 scale: e = clamp(floor(log2 amax) - 2, -127, 127); returns the E8M0 byte and
+// the exact fp32 multiplier 2^-e.  amax is finite and non-negative.
+__device__ __forceinline__ void mx_scale(float amax, uint32_t& byte, float& mult) {
+  int e = static_cast<int>((__float_as_uint(amax) >> 23) & 0xFF) - 127 - 2;   // zero/subnormal -> -129
+  e = e < -127 ? -127 : e;                                                   // e <= 125 for finite input
+  byte = static_cast<uint32_t>(e + 127);
+  mult = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);               // 2^-e, biased 2..254
+}
+
+__device__ __forceinline__ float e4m3_to_float(uint32_t byte) {
+  __half_raw h = __nv_cvt_fp8_to_halfraw(static_cast<__nv_fp8_storage_t>(byte), __NV_E4M3);
+  return __half2float(__half(h));
+}
+
+// ---- NVFP4 scale.  Single-rounded fp32 steps, in this order and with no contraction:
+//   r = (amax / 6) / ts ;  byte = E4M3(r) ;  d = float(byte) * ts ;  mult = d == 0 ? 0 : 1 / d.
+__device__ __forceinline__ void nv_scale(float amax, float ts, uint32_t& byte, float& mult) {
+  const float r = __fdiv_rn(__fdiv_rn(amax, 6.0f), ts);
+  byte = static_cast<uint32_t>(__nv_cvt_float_to_fp8(r, __NV_SATFINITE, __NV_E4M3));
+  const float d = __fmul_rn(e4m3_to_float(byte), ts);
+  mult = (d == 0.0f) ? 0.0f : __frcp_rn(d);
+}
+
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// transpose an 8x8 matrix of 16-bit elements held one 32-bit register per lane
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(y) : "r"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint4 ld_global_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+}  // namespace wush

@@ -1,0 +1,215 @@
+"""Thin ctypes binding of libwush.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/wush.h) minus the
+`wush_` prefix, takes CUDA torch tensors, allocates the output tensors with torch
+(torch is used for device memory and streams, nothing else) and enqueues the kernels
+on torch's current stream.  Nothing is computed in Python, and there is no fallback:
+if the library has not been built, or a call returns an error status, an exception
+is raised.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwush.so")
+
+MXFP4, NVFP4 = 0, 1
+SF_LINEAR, SF_TILED = 0, 1
+OUT_F32, OUT_BF16 = 0, 1
+FORMATS = {"mxfp4": (MXFP4, 32), "nvfp4": (NVFP4, 16)}
+
+EXPORTS = [
+    "wush_status_string", "wush_last_cuda_error", "wush_scale_bytes", "wush_quantize_act",
+    "wush_quantize_weight", "wush_quantize_weight_workspace_bytes", "wush_gemm_fp4", "wush_linear",
+    "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
+    "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32",
+]
+
+_lib = None
+
+
+class WushError(RuntimeError):
+    pass
+
+
+def lib():
+    """Load libwush.so once.  Raises if it is missing: there is no other code path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise WushError(f"{LIB_PATH} not found: build it with `python -m paper_2512_00956_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+        L.wush_status_string.restype = ctypes.c_char_p
+        L.wush_status_string.argtypes = [i32]
+        L.wush_last_cuda_error.restype = ctypes.c_char_p
+        L.wush_scale_bytes.restype = sz
+        L.wush_scale_bytes.argtypes = [i64, i64, i32, i32]
+        L.wush_quantize_act.argtypes = [vp, i64, i64, vp, i32, i32, vp, vp, vp, i32, vp]
+        L.wush_quantize_weight.argtypes = [vp, i64, i64, vp, i32, i32, vp, vp, vp, i32, vp, sz, vp]
+        L.wush_quantize_weight_workspace_bytes.restype = sz
+        L.wush_quantize_weight_workspace_bytes.argtypes = [i64, i64, i32, i32]
+        L.wush_gemm_fp4.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, i32, vp, vp]
+        L.wush_linear.argtypes = [vp, i64, i64, vp, vp, vp, i64, vp, vp, i32, i32, vp, i32, vp, sz, vp]
+        L.wush_linear_workspace_bytes.restype = sz
+        L.wush_linear_workspace_bytes.argtypes = [i64, i64, i32]
+        L.wush_calib_moments.argtypes = [vp, i64, i64, i32, vp, vp, vp, sz, vp]
+        L.wush_calib_moments_workspace_bytes.restype = sz
+        L.wush_calib_moments_workspace_bytes.argtypes = [i64, i64, i32]
+        L.wush_quantize_f32.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, i32, vp]
+        L.wush_transform_act_f32.argtypes = [vp, i64, i64, vp, i32, vp, vp]
+        L.wush_transform_weight_f32.argtypes = [vp, i64, i64, vp, i32, vp, vp]
+        for name in ("wush_quantize_act", "wush_quantize_weight", "wush_gemm_fp4", "wush_linear",
+                     "wush_calib_moments", "wush_quantize_f32", "wush_transform_act_f32",
+                     "wush_transform_weight_f32"):
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def check(status):
+    if status != 0:
+        L = lib()
+        msg = L.wush_status_string(status).decode()
+        if status == -6:
+            msg += ": " + L.wush_last_cuda_error().decode()
+        raise WushError(f"libwush status {status}: {msg}")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _fmt(fmt):
+    return FORMATS[fmt] if isinstance(fmt, str) else (fmt, 32 if fmt == MXFP4 else 16)
+
+
+def _dev(*ts):
+    for t in ts:
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise WushError("expected contiguous CUDA tensors")
+
+
+def scale_bytes(rows, K, g, sf):
+    return lib().wush_scale_bytes(rows, K, g, sf)
+
+
+def _alloc_q(rows, K, g, sf, device):
+    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=device)
+    nbytes = scale_bytes(rows, K, g, sf)
+    if sf == SF_LINEAR:
+        scales = torch.empty((rows, K // g), dtype=torch.uint8, device=device)
+    else:
+        scales = torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
+    return codes, scales
+
+
+def quantize_act(X, T, fmt, x_tensor_scale=None, sf=SF_LINEAR, out=None):
+    """X bf16 [M,K], T bf16 [K/g,g,g] -> (codes uint8 [M,K/2], scale bytes)."""
+    f, g = _fmt(fmt)
+    _dev(X, T, x_tensor_scale)
+    M, K = X.shape
+    codes, scales = out if out is not None else _alloc_q(M, K, g, sf, X.device)
+    check(lib().wush_quantize_act(_ptr(X), M, K, _ptr(T), f, g, _ptr(x_tensor_scale), _ptr(codes), _ptr(scales),
+                                  sf, _stream()))
+    return codes, scales
+
+
+def quantize_weight(W, Tinv, fmt, sf=SF_TILED):
+    """W bf16 [N,K], Tinv fp32 [K/g,g,g] -> (codes, scale bytes, w_tensor_scale fp32[1] or None)."""
+    f, g = _fmt(fmt)
+    _dev(W, Tinv)
+    N, K = W.shape
+    codes, scales = _alloc_q(N, K, g, sf, W.device)
+    ts = torch.zeros(4, dtype=torch.float32, device=W.device) if f == NVFP4 else None
+    nws = lib().wush_quantize_weight_workspace_bytes(N, K, f, g)
+    ws = torch.empty(nws, dtype=torch.uint8, device=W.device)
+    check(lib().wush_quantize_weight(_ptr(W), N, K, _ptr(Tinv), f, g, _ptr(ts), _ptr(codes), _ptr(scales), sf,
+                                     _ptr(ws), nws, _stream()))
+    return codes, scales, ts
+
+
+def gemm_fp4(Xq, Xs, Wq, Ws, K, fmt, x_tensor_scale=None, w_tensor_scale=None, out_dtype=torch.float32,
+             out=None, status=None):
+    """Packed codes [M,K/2], [N,K/2] + TILED scale bytes -> Y [M,N]."""
+    f, g = _fmt(fmt)
+    _dev(Xq, Xs, Wq, Ws)
+    M, N = Xq.shape[0], Wq.shape[0]
+    Y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=Xq.device)
+    ydt = OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32
+    if status is None:
+        status = torch.zeros(4, dtype=torch.int32, device=Xq.device)
+    check(lib().wush_gemm_fp4(_ptr(Xq), _ptr(Xs), _ptr(Wq), _ptr(Ws), M, N, K, f, g, _ptr(x_tensor_scale),
+                              _ptr(w_tensor_scale), _ptr(Y), ydt, _ptr(status), _stream()))
+    return Y, status
+
+
+def linear_workspace_bytes(M, K, g):
+    return lib().wush_linear_workspace_bytes(M, K, g)
+
+
+def linear(X, T, Wcodes, Wscales, fmt, x_tensor_scale=None, w_tensor_scale=None, out_dtype=torch.float32,
+           out=None, workspace=None):
+    """The whole online layer: Y = q(X T^T) (x) W~ (Eq. 7).  Returns (Y, workspace)."""
+    f, g = _fmt(fmt)
+    _dev(X, T, Wcodes, Wscales)
+    M, K = X.shape
+    N = Wcodes.shape[0]
+    Y = out if out is not None else torch.empty((M, N), dtype=out_dtype, device=X.device)
+    ydt = OUT_BF16 if Y.dtype == torch.bfloat16 else OUT_F32
+    nws = linear_workspace_bytes(M, K, g)
+    if workspace is None:
+        workspace = torch.empty(nws, dtype=torch.uint8, device=X.device)
+    check(lib().wush_linear(_ptr(X), M, K, _ptr(T), _ptr(Wcodes), _ptr(Wscales), N, _ptr(x_tensor_scale),
+                            _ptr(w_tensor_scale), f, g, _ptr(Y), ydt, _ptr(workspace), workspace.numel(), _stream()))
+    return Y, workspace
+
+
+def linear_status(workspace):
+    """The GEMM's diagnostic word kept in the last 16 bytes of a wush_linear workspace (0 = fine)."""
+    return int(workspace[-16:].view(torch.int32)[0].item())
+
+
+def calib_moments(Xc, g, moments=None, count=None):
+    """moments[c] += sum_t x_tc^T x_tc ; count += B.  Returns (moments fp32 [K/g,g,g], count int64[1])."""
+    _dev(Xc, moments, count)
+    B, K = Xc.shape
+    if moments is None:
+        moments = torch.zeros((K // g, g, g), dtype=torch.float32, device=Xc.device)
+    if count is None:
+        count = torch.zeros(2, dtype=torch.int64, device=Xc.device)
+    nws = lib().wush_calib_moments_workspace_bytes(B, K, g)
+    ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=Xc.device)
+    check(lib().wush_calib_moments(_ptr(Xc), B, K, g, _ptr(moments), _ptr(count), _ptr(ws), ws.numel(), _stream()))
+    return moments, count
+
+
+def quantize_f32(V, fmt, tensor_scale=None, sf=SF_LINEAR):
+    f, g = _fmt(fmt)
+    _dev(V, tensor_scale)
+    R, K = V.shape
+    codes, scales = _alloc_q(R, K, g, sf, V.device)
+    check(lib().wush_quantize_f32(_ptr(V), R, K, f, g, _ptr(tensor_scale), _ptr(codes), _ptr(scales), sf, _stream()))
+    return codes, scales
+
+
+def transform_act_f32(X, T, g):
+    _dev(X, T)
+    M, K = X.shape
+    V = torch.empty((M, K), dtype=torch.float32, device=X.device)
+    check(lib().wush_transform_act_f32(_ptr(X), M, K, _ptr(T), g, _ptr(V), _stream()))
+    return V
+
+
+def transform_weight_f32(W, Tinv, g):
+    _dev(W, Tinv)
+    N, K = W.shape
+    V = torch.empty((N, K), dtype=torch.float32, device=W.device)
+    check(lib().wush_transform_weight_f32(_ptr(W), N, K, _ptr(Tinv), g, _ptr(V), _stream()))
+    return V

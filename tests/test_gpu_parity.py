@@ -1,0 +1,202 @@
+"""GPU parity tests: every entry point of libwush against the CPU oracle on the same
+seeded inputs, called through the C ABI (ctypes binding).  Sizes span several tiles and
+ragged tails; tolerances are the build target's:
+  - stand-alone quantiser on fp32 input: codes and scale bytes bit-exact;
+  - transform: |v_gpu - v_oracle| <= 1e-5 * AbsMax(block);
+  - transform + quantise: bit-exact outside the 1e-4 guard bands, one step inside;
+  - Y: relative Frobenius error <= 1e-3 (fp32 output);  moments: <= 1e-5.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import formats as F
+from oracle import pipeline as P
+from oracle import quantizers as Q
+from paper_2512_00956_b200 import synth, wush
+from parity_util import (compare_quantized, dev, dev_bf16, rel_fro, tile, untile)
+
+pytestmark = pytest.mark.gpu
+G = Q.GROUP
+
+
+def _sync():
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ stand-alone quantiser
+def _quantizer_inputs(fmt, R, K, seed):
+    rng = np.random.default_rng(seed)
+    g = G[fmt]
+    spread = 20 if fmt == "mxfp4" else 3
+    v = (rng.standard_normal((R, K)) * np.exp(rng.uniform(-spread, spread, (R, K // g, 1)).repeat(g, 2).reshape(R, K)))
+    v = v.astype(np.float32)
+    v[0, :g] = 0.0                                            # all-zero block
+    v[1, :g] = -0.0
+    mids = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 4.0, -0.25, -5.0], dtype=np.float32)
+    v[2, :g] = 0; v[2, :len(mids)] = mids                     # exact ties, block AbsMax 6 -> scale 1
+    v[3, :g] = np.float32(2.0 ** 5) * (1 - 2.0 ** -24)        # just under a power of two
+    v[4, :g] = 1e-38 if fmt == "mxfp4" else 1e-6              # tiny / subnormal scale region
+    v[5, :g] = 3e38 if fmt == "mxfp4" else 1e4                # huge (NVFP4: saturating scale)
+    return v
+
+
+@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4"])
+@pytest.mark.parametrize("sf", [wush.SF_LINEAR, wush.SF_TILED])
+def test_quantize_f32_bit_exact(fmt, sf):
+    R, K = 333, 512
+    v = _quantizer_inputs(fmt, R, K, 11)
+    ts = np.float32(0.0371) if fmt == "nvfp4" else None
+    ts_d = dev(np.full(4, ts, dtype=np.float32)) if ts is not None else None
+    codes, scales = wush.quantize_f32(dev(v), fmt, ts_d, sf)
+    _sync()
+    sc = scales.cpu().numpy()
+    if sf == wush.SF_TILED:
+        sc = untile(sc, R, K // G[fmt])
+    compare_quantized(codes.cpu().numpy(), sc, v, fmt, ts, strict=True)
+
+
+# ------------------------------------------------------------------ transform alone
+def _layer(idx, fmt, M=None, N=None, K=None, B=None):
+    cfg = synth.CONFIGS[idx]
+    d = synth.layer_inputs(cfg, M=M, N=N, K=K, B=B)
+    return d, P.PreparedLayer(d["W"], d["Xc"], fmt)
+
+
+@pytest.mark.parametrize("fmt,M,K", [("mxfp4", 128, 2048), ("nvfp4", 77, 320), ("mxfp4", 1, 64), ("nvfp4", 300, 1024)])
+def test_transform_act_f32(fmt, M, K):
+    d, L = _layer(1, fmt, M=M, N=64, K=K, B=256)
+    g = G[fmt]
+    V = wush.transform_act_f32(dev_bf16(d["X"]), dev_bf16(L.T_bits), g)
+    _sync()
+    v_o = P.transform_blocks(F.bf16_bits_to_f64(d["X"]), L.T_hat)
+    amax = np.abs(v_o.reshape(M, K // g, g)).max(axis=2).repeat(g, axis=1)
+    err = np.abs(V.cpu().numpy().astype(np.float64) - v_o)
+    assert np.all(err <= 1e-5 * amax + 1e-300), float((err / np.maximum(amax, 1e-300)).max())
+
+
+@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4"])
+def test_transform_weight_f32(fmt):
+    d, L = _layer(1, fmt, M=16, N=200, K=384, B=256)
+    g = G[fmt]
+    V = wush.transform_weight_f32(dev_bf16(d["W"]), dev(L.T_xvsh32), g)
+    _sync()
+    w_o = P.transform_blocks(F.bf16_bits_to_f64(d["W"]), L.T_xvsh32.astype(np.float64))
+    amax = np.abs(w_o.reshape(200, 384 // g, g)).max(axis=2).repeat(g, axis=1)
+    err = np.abs(V.cpu().numpy().astype(np.float64) - w_o)
+    assert np.all(err <= 1e-5 * amax), float((err / amax).max())
+
+
+# ------------------------------------------------------------------ transform + quantise
+@pytest.mark.parametrize("fmt,M,K,sf", [
+    ("mxfp4", 128, 2048, wush.SF_LINEAR), ("mxfp4", 77, 192, wush.SF_LINEAR), ("mxfp4", 1, 64, wush.SF_TILED),
+    ("mxfp4", 300, 1024, wush.SF_TILED), ("nvfp4", 128, 2048, wush.SF_LINEAR), ("nvfp4", 77, 320, wush.SF_TILED),
+    ("nvfp4", 16, 64, wush.SF_LINEAR), ("nvfp4", 531, 1024, wush.SF_TILED)])
+def test_quantize_act_parity(fmt, M, K, sf):
+    d, L = _layer(1 if fmt == "mxfp4" else 2, fmt, M=M, N=64, K=K, B=256)
+    ts_d = dev(np.full(4, L.ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
+    codes, scales = wush.quantize_act(dev_bf16(d["X"]), dev_bf16(L.T_bits), fmt, ts_d, sf)
+    _sync()
+    sc = scales.cpu().numpy()
+    if sf == wush.SF_TILED:
+        sc = untile(sc, M, K // G[fmt])
+    v32, _, _ = L.quantize_act(d["X"])
+    stats = compare_quantized(codes.cpu().numpy(), sc, v32, fmt, L.ts_x)
+    assert stats["flipped_codes"] <= stats["guarded_elems"]
+
+
+def test_quantize_act_deterministic_and_in_bounds():
+    d, L = _layer(1, "mxfp4", M=200, N=64, K=512, B=256)
+    X, T = dev_bf16(d["X"]), dev_bf16(L.T_bits)
+    pad = 4096
+    codes = torch.full((200 * 256 + 2 * pad,), 0xAB, dtype=torch.uint8, device="cuda")
+    scales = torch.full((200 * 16 + 2 * pad,), 0xCD, dtype=torch.uint8, device="cuda")
+    out = (codes[pad:pad + 200 * 256].view(200, 256), scales[pad:pad + 200 * 16].view(200, 16))
+    wush.quantize_act(X, T, "mxfp4", None, wush.SF_LINEAR, out=out)
+    c1, s1 = out[0].clone(), out[1].clone()
+    wush.quantize_act(X, T, "mxfp4", None, wush.SF_LINEAR, out=out)
+    _sync()
+    assert torch.equal(c1, out[0]) and torch.equal(s1, out[1])
+    for buf, val, n in ((codes, 0xAB, 200 * 256), (scales, 0xCD, 200 * 16)):     # canaries untouched
+        assert bool((buf[:pad] == val).all()) and bool((buf[pad + n:] == val).all())
+
+
+# ------------------------------------------------------------------ weight side
+@pytest.mark.parametrize("fmt,N,K", [("mxfp4", 200, 384), ("nvfp4", 200, 384), ("mxfp4", 2048, 2048), ("nvfp4", 1000, 1024)])
+def test_quantize_weight_parity(fmt, N, K):
+    d, L = _layer(1, fmt, M=16, N=N, K=K, B=256)
+    codes, scales, ts = wush.quantize_weight(dev_bf16(d["W"]), dev(L.T_xvsh32), fmt, sf=wush.SF_LINEAR)
+    _sync()
+    if fmt == "nvfp4":
+        ts_g = float(ts.cpu().numpy()[0])
+        assert abs(ts_g - float(L.ts_w)) <= 2e-7 * float(L.ts_w)
+    compare_quantized(codes.cpu().numpy(), scales.cpu().numpy(), L.wbar32, fmt, L.ts_w)
+
+
+# ------------------------------------------------------------------ moments
+@pytest.mark.parametrize("g,B,K", [(32, 512, 2048), (16, 333, 320), (32, 1, 64), (16, 1024, 4096)])
+def test_calib_moments(g, B, K):
+    cfg = synth.CONFIGS[1]
+    Xc = synth.calibration(cfg, B=B, K=K)
+    mom, cnt = wush.calib_moments(dev_bf16(Xc), g)
+    _sync()
+    S = P.second_moment_sums(F.bf16_bits_to_f64(Xc), g)
+    assert rel_fro(mom.cpu().numpy(), S) <= 1e-5
+    assert int(cnt[0].item()) == B
+    # accumulate in place: a second chunk adds on top, bit-identically from run to run
+    mom2, cnt2 = wush.calib_moments(dev_bf16(Xc), g, mom.clone(), cnt.clone())
+    mom3, _ = wush.calib_moments(dev_bf16(Xc), g, mom.clone(), cnt.clone())
+    _sync()
+    assert int(cnt2[0].item()) == 2 * B and torch.equal(mom2, mom3)
+    assert rel_fro(mom2.cpu().numpy(), 2 * S) <= 1e-5
+
+
+# ------------------------------------------------------------------ GEMM alone (oracle's codes in)
+@pytest.mark.parametrize("fmt,M,N,K", [
+    ("mxfp4", 128, 256, 256), ("mxfp4", 3, 8, 64), ("mxfp4", 200, 264, 448), ("mxfp4", 128, 2048, 2048),
+    ("nvfp4", 128, 256, 256), ("nvfp4", 5, 16, 64), ("nvfp4", 131, 392, 320), ("nvfp4", 300, 1024, 1536)])
+def test_gemm_fp4_against_oracle_product(fmt, M, N, K):
+    d, L = _layer(1, fmt, M=M, N=N, K=K, B=256)
+    g = G[fmt]
+    _, xc, xs = L.quantize_act(d["X"])
+    Y_o = P.dequantized_product(Q.dequantize(xc, xs, fmt, L.ts_x), L.w_deq)
+    tsx = dev(np.full(4, L.ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
+    tsw = dev(np.full(4, L.ts_w, dtype=np.float32)) if fmt == "nvfp4" else None
+    Y, status = wush.gemm_fp4(dev(F.pack_e2m1(xc)), dev(tile(xs)), dev(F.pack_e2m1(L.w_codes)), dev(tile(L.w_scales)),
+                              K, fmt, tsx, tsw)
+    _sync()
+    assert int(status[0].item()) == 0, hex(int(status[0].item()))
+    assert rel_fro(Y.cpu().numpy(), Y_o) <= 1e-5                      # same codes in: only fp32 accumulation differs
+    Yb, _ = wush.gemm_fp4(dev(F.pack_e2m1(xc)), dev(tile(xs)), dev(F.pack_e2m1(L.w_codes)), dev(tile(L.w_scales)),
+                          K, fmt, tsx, tsw, out_dtype=torch.bfloat16)
+    _sync()
+    Y_ob = F.round_to_bf16(Y_o)
+    assert rel_fro(Yb.float().cpu().numpy(), Y_ob) <= 4e-3            # bf16 output vs bf16-rounded oracle
+
+
+# ------------------------------------------------------------------ the whole layer
+def _run_linear(idx, fmt, M=None, N=None, K=None, B=None, rows=None):
+    d, L = _layer(idx, fmt, M=M, N=N, K=K, B=B)
+    g = G[fmt]
+    W, X = dev_bf16(d["W"]), dev_bf16(d["X"])
+    wq, ws, tsw = wush.quantize_weight(W, dev(L.T_xvsh32), fmt, sf=wush.SF_TILED)
+    tsx = dev(np.full(4, L.ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
+    Y, wsp = wush.linear(X, dev_bf16(L.T_bits), wq, ws, fmt, tsx, tsw)
+    _sync()
+    assert wush.linear_status(wsp) == 0
+    Yg = Y.cpu().numpy()
+    Y_o = L.forward(d["X"], rows=rows)
+    return rel_fro(Yg if rows is None else Yg[rows], Y_o)
+
+
+@pytest.mark.parametrize("fmt,M,N,K", [("mxfp4", 77, 136, 320), ("nvfp4", 77, 136, 320), ("mxfp4", 260, 520, 1024)])
+def test_linear_small(fmt, M, N, K):
+    assert _run_linear(1, fmt, M=M, N=N, K=K, B=256) <= 1e-3
+
+
+def test_linear_config1_full():
+    assert _run_linear(1, "mxfp4") <= 1e-3
+
+
+def test_linear_config2_full():
+    assert _run_linear(2, "nvfp4") <= 1e-3
