@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the online W4A4 WUSH linear layer (Eq. 7) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+
+A step is one pass of the whole hot path - fused transform + quantise of X, then the
+block-scaled FP4 GEMM against the pre-quantised weights - over one batch of synthetic tokens
+(`wush_linear`).  Rank 0 prints ONE JSON line.  `value` is 2*M*N*K / step time summed over
+ranks (each rank runs its own replica of the layer on its own tokens: weak scaling, no
+data-path collective).  The line also carries the roofline of the dominant kernel, the
+quantiser's HBM figure, the cuBLAS bf16 GEMM of the same shape, an end-to-end number with
+host buffers, sampled clocks, and the CPU oracle timed on the host cores.
+
+`--impl reference` times the CPU oracle (the only "reference" this method has here).
+"""
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "W4A4 WUSH linear TFLOP/s (2MNK / step time; transform+quant + FP4 GEMM)"
+
+
+def load_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    except Exception:
+        return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def pick_config(args):
+    from paper_2512_00956_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    fmt = args.fmt or cfg.formats[0]
+    M = args.m or cfg.M
+    return cfg, fmt, M
+
+
+def oracle_sample_seconds(cfg, fmt, M, rows):
+    """Times the CPU oracle's online path (transform, quantise, dequantised product) on `rows` tokens."""
+    from oracle import pipeline as P
+    from paper_2512_00956_b200 import synth
+    d = synth.layer_inputs(cfg, M=rows)
+    L = P.PreparedLayer(d["W"], d["Xc"], fmt)            # offline part, not timed
+    t0 = time.perf_counter()
+    L.forward(d["X"])
+    return time.perf_counter() - t0
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, fmt, M = pick_config(args)
+    from oracle import pipeline as P
+    from paper_2512_00956_b200 import synth
+    rows = min(M, args.ref_rows)
+    d = synth.layer_inputs(cfg, M=rows)
+    L = P.PreparedLayer(d["W"], d["Xc"], fmt)
+    for _ in range(args.warmup):
+        L.forward(d["X"])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        L.forward(d["X"])
+    dt = (time.perf_counter() - t0) / args.steps
+    tf = 2.0 * rows * cfg.N * cfg.K / dt / 1e12
+    sample = f"{rows} of {M} token rows x all N={cfg.N}, K={cfg.K} per step (fp64 numpy)"
+    line = {"impl": "reference", "metric": METRIC, "value": tf, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "M": M, "K": cfg.K, "N": cfg.N, "format": fmt, "sample_rows": rows},
+            "cpu_baseline": {"value": tf, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": tf, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2512_00956_b200 import dist as D
+    from paper_2512_00956_b200 import prepare, synth, wush
+
+    rank, local_rank, world = D.init()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    wush.lib()                                           # fail loudly if the library is missing
+    peaks = load_peaks()
+    cfg, fmt, M = pick_config(args)
+    g = synth.GROUP[fmt]
+    K, N = cfg.K, cfg.N
+    out_dtype = torch.bfloat16 if args.out == "bf16" else torch.float32
+
+    def up(bits):
+        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(dev)
+
+    Xh_bits = synth.activations(cfg, M=M)
+    W, Xc = up(synth.weights(cfg)), up(synth.calibration(cfg))
+    layer = prepare.QuantizedLinear(W, Xc, fmt)
+    X = up(Xh_bits)
+    Y = torch.empty((M, N), dtype=out_dtype, device=dev)
+    ws = torch.empty(wush.linear_workspace_bytes(M, K, g), dtype=torch.uint8, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)          # > L2 (126 MB)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        wush.linear(X, layer.T, layer.w_codes, layer.w_scales, fmt, layer.x_tensor_scale, layer.w_tensor_scale,
+                    out=Y, workspace=ws)
+
+    xq = ws[: M * K // 2].view(M, K // 2)
+    xs = ws[(M * K // 2 + 15) // 16 * 16:][: wush.scale_bytes(M, K, g, wush.SF_TILED)]
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+
+    def step_split(evs):
+        evs[0].record(stream)
+        wush.quantize_act(X, layer.T, fmt, layer.x_tensor_scale, wush.SF_TILED, out=(xq, xs))
+        evs[1].record(stream)
+        wush.gemm_fp4(xq, xs, layer.w_codes, layer.w_scales, K, fmt, layer.x_tensor_scale, layer.w_tensor_scale,
+                      out=Y, status=status)
+        evs[2].record(stream)
+
+    for _ in range(max(3, args.warmup)):
+        flush.zero_()
+        step()
+    torch.cuda.synchronize()
+
+    # ---- timed region: exactly K steps, cold L2 (a 512 MB write between steps, outside the event pairs)
+    sampler = ClockSampler(local_rank)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    D.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    wall0 = time.perf_counter()
+    for a, b in ev:
+        flush.zero_()
+        a.record(stream)
+        step()
+        b.record(stream)
+    torch.cuda.synchronize()
+    D.barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop()
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    ms_rank = sum(step_ms) / len(step_ms)
+    gemm_status = wush.linear_status(ws, M, K, g)
+
+    # ---- per-kernel durations (same launches, issued separately so events can sit between them)
+    ev3 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for e in ev3:
+        flush.zero_()
+        step_split(e)
+    torch.cuda.synchronize()
+    q_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev3)
+    g_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev3)
+
+    # ---- cuBLAS bf16 GEMM of the same shape (the paper's normaliser), same protocol
+    Yb = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    evb = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for _ in range(3):
+        torch.matmul(X, W.t(), out=Yb)
+    for a, b in evb:
+        flush.zero_()
+        a.record(stream)
+        torch.matmul(X, W.t(), out=Yb)
+        b.record(stream)
+    torch.cuda.synchronize()
+    bf16_ms = statistics.mean(a.elapsed_time(b) for a, b in evb)
+
+    # ---- end to end through the public call with HOST buffers: pinned X in, Y back out, every step
+    Xh = torch.from_numpy(Xh_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Yh = torch.empty((M, N), dtype=out_dtype).pin_memory()
+    n_e2e = max(5, min(args.steps, 50))
+    for _ in range(2):
+        X.copy_(Xh, non_blocking=True); step(); Yh.copy_(Y, non_blocking=True)
+    torch.cuda.synchronize()
+    D.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(n_e2e):
+        X.copy_(Xh, non_blocking=True)
+        step()
+        Yh.copy_(Y, non_blocking=True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms_rank = e0.elapsed_time(e1) / n_e2e
+
+    flops = 2.0 * M * N * K
+    rate, t_max = D.whole_job_rate(flops, ms_rank * 1e-3, dev)
+    e2e_rate, _ = D.whole_job_rate(flops, e2e_ms_rank * 1e-3, dev)
+    D.barrier()
+    if rank != 0:
+        D.shutdown()
+        return
+
+    # ---- rooflines.  Dominant kernel: the FP4 GEMM (dense contraction -> tensor peak for FP4 =
+    # measured bf16 burst peak x nominal FP4:bf16 ratio 4).  Quantiser: HBM.
+    fp4_peak = peaks["bf16_tflops"] * 4.0
+    gemm_tf = flops / (g_ms * 1e-3) / 1e12
+    q_bytes = 2.0 * M * K + M * K / 2.0 + M * K / g + 2.0 * K * g
+    q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
+    roof = {"bound": "tensor", "kernel": "gemm_fp4_kernel", "achieved": gemm_tf, "peak": fp4_peak, "unit": "TFLOP/s",
+            "frac": gemm_tf / fp4_peak, "traffic": None, "ms": g_ms,
+            "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TF/s x 4 (nominal FP4:bf16)",
+            "frac_of_spec_9pf": gemm_tf / 9000.0}
+    roof_q = {"bound": "hbm", "kernel": "transform_quant_kernel", "achieved": q_gbs, "peak": peaks["hbm_gbs"],
+              "unit": "GB/s", "frac": q_gbs / peaks["hbm_gbs"], "traffic": None, "ms": q_ms,
+              "algorithmic_bytes": q_bytes, "peak_source": peaks["source"], "frac_of_spec_8tbs": q_gbs / 8000.0}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        rows = min(M, args.ref_rows)
+        sec = oracle_sample_seconds(cfg, fmt, M, rows)
+        cpu = {"value": 2.0 * rows * N * K / sec / 1e12, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
+               "sample": f"{rows} of {M} token rows x all N, one pass of the online path (fp64 numpy), {sec:.2f} s"}
+
+    line = {"metric": METRIC, "value": rate / 1e12, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": t_max * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
+            "config": {"workload": cfg.name, "M": M, "K": K, "N": N, "format": fmt, "g": g, "y_dtype": args.out,
+                       "l2": "cold: 512 MB written between timed steps", "tokens_per_rank": M},
+            "roofline": roof, "roofline_quant": roof_q,
+            "bf16_gemm": {"ms": bf16_ms, "tflops": flops / (bf16_ms * 1e-3) / 1e12, "speedup_linear": bf16_ms / ms_rank,
+                          "speedup_gemm_only": bf16_ms / g_ms, "impl": "torch.matmul (cuBLAS)"},
+            "e2e": {"value": e2e_rate / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": int(X.numel() * 2),
+                    "d2h_bytes_per_step": int(Y.numel() * Y.element_size()), "ms_per_step": e2e_ms_rank},
+            "gpu_launches": 2 * args.steps, "kernel_ms": {"transform_quant": q_ms, "gemm_fp4": g_ms},
+            "gemm_status": gemm_status, "clocks": clocks, "wall_s_timed_region": wall, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    D.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload index 1..5 (2 = the headline configuration)")
+    ap.add_argument("--fmt", default=None, choices=[None, "mxfp4", "nvfp4"])
+    ap.add_argument("--m", type=int, default=None, help="override the token count (config 5 sweep)")
+    ap.add_argument("--out", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--ref-rows", type=int, default=2048, help="token rows in the CPU-oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -123,8 +123,8 @@ int wush_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const
 
 /* The whole online layer (Eq. 7): wush_quantize_act into `workspace`, then wush_gemm_fp4,
  * both on `stream`.  Wcodes/Wscales come from wush_quantize_weight with WUSH_SF_TILED.
- * workspace: at least wush_linear_workspace_bytes(M, K, g) bytes, 16-byte aligned.  Its
- * last 16 bytes receive the GEMM's status word (see wush_gemm_fp4). */
+ * workspace: at least wush_linear_workspace_bytes(M, K, g) bytes, 16-byte aligned.  The
+ * last 16 bytes of that region receive the GEMM's status word (see wush_gemm_fp4). */
 int wush_linear(const void* X, int64_t M, int64_t K, const void* T,
                 const uint8_t* Wcodes, const uint8_t* Wscales, int64_t N,
                 const float* x_tensor_scale, const float* w_tensor_scale,

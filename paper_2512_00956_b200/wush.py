@@ -171,9 +171,11 @@ def linear(X, T, Wcodes, Wscales, fmt, x_tensor_scale=None, w_tensor_scale=None,
     return Y, workspace
 
 
-def linear_status(workspace):
-    """The GEMM's diagnostic word kept in the last 16 bytes of a wush_linear workspace (0 = fine)."""
-    return int(workspace[-16:].view(torch.int32)[0].item())
+def linear_status(workspace, M, K, g):
+    """The GEMM's diagnostic word, kept in the last 16 bytes of the wush_linear_workspace_bytes(M, K, g)
+    region of the workspace (0 = no bounded wait expired).  Synchronises."""
+    end = linear_workspace_bytes(M, K, g)
+    return int(workspace[end - 16:end].view(torch.int32)[0].item())
 
 
 def calib_moments(Xc, g, moments=None, count=None):

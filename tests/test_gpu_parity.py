@@ -183,7 +183,7 @@ def _run_linear(idx, fmt, M=None, N=None, K=None, B=None, rows=None):
     tsx = dev(np.full(4, L.ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
     Y, wsp = wush.linear(X, dev_bf16(L.T_bits), wq, ws, fmt, tsx, tsw)
     _sync()
-    assert wush.linear_status(wsp) == 0
+    assert wush.linear_status(wsp, X.shape[0], X.shape[1], g) == 0
     Yg = Y.cpu().numpy()
     Y_o = L.forward(d["X"], rows=rows)
     return rel_fro(Yg if rows is None else Yg[rows], Y_o)
@@ -200,3 +200,46 @@ def test_linear_config1_full():
 
 def test_linear_config2_full():
     assert _run_linear(2, "nvfp4") <= 1e-3
+
+
+# ------------------------------------------------------------------ GPU-side layer preparation
+@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4"])
+def test_prepare_layer_invariants_and_loss_level(fmt):
+    """The product-side transform builder is checked by invariants (several T are equally valid),
+    and the layer it prepares must reach the oracle's quantisation-error level."""
+    from paper_2512_00956_b200 import prepare
+    cfg = synth.CONFIGS[1]
+    d = synth.layer_inputs(cfg, M=128, N=256, K=512, B=512)
+    g = G[fmt]
+    W, Xc, X = dev_bf16(d["W"]), dev_bf16(d["Xc"]), dev_bf16(d["X"])
+    layer = prepare.QuantizedLinear(W, Xc, fmt)
+    _sync()
+    T = layer.T.double().cpu().numpy(); Tinv = layer.Tinv.double().cpu().numpy()
+    for c in range(T.shape[0]):
+        assert np.allclose(Tinv[c] @ T[c].T, np.eye(g), atol=1e-5)                 # Eq. 6 on the stored values
+    Xcv = F.bf16_bits_to_f64(d["Xc"])
+    mX = P.second_moment_sums(Xcv, g) / Xcv.shape[0]
+    for c in range(0, T.shape[0], 5):                                              # equalised diagonal (appendix)
+        A = T[c] @ (mX[c] + 0.01 * np.trace(mX[c]) / g * np.eye(g)) @ T[c].T
+        assert np.ptp(np.diag(A)) <= 0.05 * np.diag(A).mean()
+    Y = layer(X).cpu().numpy()
+    Xv, Wv = F.bf16_bits_to_f64(d["X"]), F.bf16_bits_to_f64(d["W"])
+    Y0 = Xv @ Wv.T
+    L = P.PreparedLayer(d["W"], d["Xc"], fmt)
+    loss_gpu = rel_fro(Y, Y0); loss_oracle = rel_fro(L.forward(d["X"]), Y0)
+    assert abs(loss_gpu - loss_oracle) <= 0.1 * loss_oracle, (loss_gpu, loss_oracle)
+    # the oracle's transforms and the GPU-built ones agree closely (same conventions)
+    assert np.abs(T - L.T_hat).max() <= 0.02 * np.abs(L.T_hat).max()
+
+
+def test_linear_bf16_output_config2_bench_configuration():
+    """The configuration bench.py times by default: config 2, NVFP4, bf16 output."""
+    d, L = _layer(2, "nvfp4")
+    W, X = dev_bf16(d["W"]), dev_bf16(d["X"])
+    wq, ws, tsw = wush.quantize_weight(W, dev(L.T_xvsh32), "nvfp4", sf=wush.SF_TILED)
+    tsx = dev(np.full(4, L.ts_x, dtype=np.float32))
+    Y, wsp = wush.linear(X, dev_bf16(L.T_bits), wq, ws, "nvfp4", tsx, tsw, out_dtype=torch.bfloat16)
+    _sync()
+    assert wush.linear_status(wsp, X.shape[0], X.shape[1], 16) == 0
+    Yo = F.round_to_bf16(L.forward(d["X"]))
+    assert rel_fro(Y.float().cpu().numpy(), Yo) <= 1e-3
