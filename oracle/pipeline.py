@@ -62,7 +62,7 @@ class PreparedLayer:
         self.mom_X = second_moment_sums(Xc, g) / Xc.shape[0]
         self.T_bits, self.T_hat, T_xvsh = WT.build_transforms(self.mom_W, self.mom_X, lam)
         # the GPU library receives the weight-side transform as fp32
-        self.T_xvsh32 = T_xvsh.astype(F32)
+        self.T_xvsh32 = np.ascontiguousarray(T_xvsh, dtype=F32)
         wbar = transform_blocks(Wv, self.T_xvsh32.astype(np.float64))
         self.wbar32 = wbar.astype(F32)
         if fmt == "nvfp4":

@@ -78,7 +78,7 @@ def build_transforms(mom_W, mom_X, lam=0.01):
     T = np.stack([wush_block(mom_W[c], mom_X[c], lam) for c in range(C)])
     bits = F.f64_to_bf16_bits(T)
     That = F.bf16_bits_to_f64(bits)
-    Tx = np.stack([xvsh_from_wush(That[c]) for c in range(C)])
+    Tx = np.ascontiguousarray(np.stack([xvsh_from_wush(That[c]) for c in range(C)]))
     return bits, That, Tx
 
 
