@@ -88,6 +88,12 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
       : "memory");
 }
+// true in exactly one lane of a fully converged warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -192,61 +198,72 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------------------------------------------ operand producer
-    if (lane == 0) {
-      int issued = 0;
-      bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag)) {
+    // The whole warp walks the loop (warp-uniform control flow keeps addresses and descriptors in
+    // uniform registers); one elected lane issues the copies.
+    int issued = 0;
+    bool ok = true;
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % STAGES;
+      const uint32_t ph = (kb / STAGES) & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag))) {
+        if (lane == 0) {
           if (*abort_flag == 0 && status) atomicExch(status, 0x10000 | kb);
-          *abort_flag = 1; ok = false; break;
+          *abort_flag = 1;
         }
-        const int tiles = min(TPS, ktiles_total - kb * TPS);
-        const bool grp1 = (n0 + 128) < ((N + 127) & ~127);      // second 128-row scale group exists
-        const uint32_t sf_bytes = tiles * 512;
-        const uint32_t bar = smem_u32(&full_bar[s]);
+        ok = false;
+        break;
+      }
+      const int tiles = min(TPS, ktiles_total - kb * TPS);
+      const bool grp1 = (n0 + 128) < ((N + 127) & ~127);      // second 128-row scale group exists
+      const uint32_t sf_bytes = tiles * 512;
+      const uint32_t bar = smem_u32(&full_bar[s]);
+      uint8_t* sf = sSF + s * stage_sf_bytes(FMT);
+      if (elect_one()) {
         mbar_expect_tx(bar, A_BYTES + B_BYTES + sf_bytes * (grp1 ? 3 : 2));
         tma_load_2d(smem_u32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
         tma_load_2d(smem_u32(sB + s * B_BYTES), &mapB, kb * BKB, n0, bar);
-        uint8_t* sf = sSF + s * stage_sf_bytes(FMT);
         bulk_load_1d(smem_u32(sf), SFA + ((int64_t)(m0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
         bulk_load_1d(smem_u32(sf + TPS * 512), SFB + ((int64_t)(n0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
         if (grp1)
           bulk_load_1d(smem_u32(sf + 2 * TPS * 512), SFB + ((int64_t)((n0 >> 7) + 1) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
-        ++issued;
       }
-      if (!ok) {
-        // drain: every stage filled must land before the CTA may exit
-        for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
-          const uint64_t t0 = global_timer_ns();
-          while (!mbar_try_wait(smem_u32(&full_bar[kb % STAGES]), (kb / STAGES) & 1))
-            if (global_timer_ns() - t0 > 500000000ull) break;
-        }
+      __syncwarp();
+      ++issued;
+    }
+    if (!ok) {
+      // drain: every stage filled must land before the CTA may exit
+      for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
+        const uint64_t t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&full_bar[kb % STAGES]), (kb / STAGES) & 1))
+          if (global_timer_ns() - t0 > 500000000ull) break;
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag)) {
+    bool ok = true;
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % STAGES;
+      const uint32_t ph = (kb / STAGES) & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag))) {
+        if (lane == 0) {
           if (*abort_flag == 0 && status) atomicExch(status, 0x20000 | kb);
-          *abort_flag = 1; ok = false; break;
+          *abort_flag = 1;
         }
-        tc_fence_after();
-        const int tiles = min(TPS, ktiles_total - kb * TPS);
-        const uint32_t sf = smem_u32(sSF + s * stage_sf_bytes(FMT));
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const int tiles = min(TPS, ktiles_total - kb * TPS);
+      const uint32_t sf = smem_u32(sSF + s * stage_sf_bytes(FMT));
+      const int ksteps = min(4, (K - kb * 2 * BKB) / 64);
+      const uint64_t adesc = operand_desc(smem_u32(sA + s * A_BYTES));
+      const uint64_t bdesc = operand_desc(smem_u32(sB + s * B_BYTES));
+      if (elect_one()) {
         for (int i = 0; i < tiles; ++i) {
           tc_cp_sf(tmem_base + SFA_COL + 4 * i, scale_desc(sf + i * 512));
           tc_cp_sf(tmem_base + SFB_COL + 8 * i, scale_desc(sf + (TPS + i) * 512));
           tc_cp_sf(tmem_base + SFB_COL + 8 * i + 4, scale_desc(sf + (2 * TPS + i) * 512));
         }
-        const int ksteps = min(4, (K - kb * 2 * BKB) / 64);
-        const uint64_t adesc = operand_desc(smem_u32(sA + s * A_BYTES));
-        const uint64_t bdesc = operand_desc(smem_u32(sB + s * B_BYTES));
         for (int j = 0; j < ksteps; ++j) {
           const int tile = j / KSTEPS_PER_TILE;
           const uint32_t sf_byte = (FMT == kFmtMX) ? 2u * (j % KSTEPS_PER_TILE) : 0u;
@@ -255,12 +272,14 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         }
         tc_commit(smem_u32(&empty_bar[s]));
       }
-      tc_commit(smem_u32(tmem_full_bar));
-      if (!ok) {   // let outstanding MMAs finish before tensor memory is released
-        const uint64_t t0 = global_timer_ns();
-        while (!mbar_try_wait(smem_u32(tmem_full_bar), 0))
-          if (global_timer_ns() - t0 > 500000000ull) break;
-      }
+      __syncwarp();
+    }
+    if (elect_one()) tc_commit(smem_u32(tmem_full_bar));
+    __syncwarp();
+    if (!ok) {   // let outstanding MMAs finish before tensor memory is released
+      const uint64_t t0 = global_timer_ns();
+      while (!mbar_try_wait(smem_u32(tmem_full_bar), 0))
+        if (global_timer_ns() - t0 > 500000000ull) break;
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
