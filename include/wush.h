@@ -144,6 +144,33 @@ int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* momen
                        int64_t* count, void* workspace, size_t workspace_bytes, void* stream);
 size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g);
 
+/* wush_calib_moments without a workspace argument.  (No counterpart in the paper: this is
+ * a packaging variant of the call above, added for hosts where this library must not and
+ * cannot obtain device memory at call time - for example a serving process whose allocator
+ * has claimed the whole HBM for its own arena and has no API to lend a slice to a plug-in,
+ * or a runtime that forbids allocation after start-up.  Such a caller has nowhere to get
+ * the scratch buffer the normal entry point asks for.)
+ *
+ * The per-split partial sums live in a fixed array of WUSH_STATIC_SCRATCH_BYTES inside the
+ * library image; every GPU that loads the library carries that array until the process
+ * exits.  Inputs and outputs are still the caller's.  The call allocates nothing and frees
+ * nothing.  Limits and rules:
+ *   - K * g * 4 bytes (one set of partial sums) must fit in the array, otherwise
+ *     WUSH_ERR_WORKSPACE is returned and nothing is launched; larger B only lowers the number
+ *     of token splits that run in parallel (down to one), never the result;
+ *   - the first call on each device resolves the array's device address (a CUDA runtime
+ *     symbol lookup, done once per device with that device current); make that first call
+ *     during start-up, before any stream capture;
+ *   - all calls on a device share the one array.  It keeps whatever the previous call left;
+ *     nothing in it needs clearing because every call overwrites the part it reads.  Two
+ *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it:
+ *     serialise them;
+ *   - results match wush_calib_moments to fp32 summation-order differences (identical when
+ *     both use the same number of splits), and are run-to-run identical. */
+#define WUSH_STATIC_SCRATCH_BYTES (4u << 20)
+int wush_calib_moments_static(const void* Xc, int64_t B, int64_t K, int g, float* moments,
+                              int64_t* count, void* stream);
+
 /* ----------------------------------------------------------------- diagnostic exports */
 /* The block quantiser q(.) alone on fp32 input V[R,K] (same outputs as above). */
 int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, int g,

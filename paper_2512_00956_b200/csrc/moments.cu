@@ -8,6 +8,9 @@
 // the 32x32 outer-product sum with mma.sync (bf16 products are exact in fp32).  Token ranges
 // are split over CTAs; the per-split partial sums go to a workspace and a second kernel adds
 // them in a fixed order, so the result does not depend on scheduling.
+#include <mutex>
+
+#include "../../include/wush.h"
 #include "wush_device.cuh"
 #include "wush_host.h"
 
@@ -116,3 +119,58 @@ cudaError_t run_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float
 }
 
 }  // namespace wush
+
+// ------------------------------------------------------------------------------------------
+// wush_calib_moments_static: the same computation with the per-split partial sums kept in a
+// fixed device array that is part of the library image, for callers that cannot supply
+// scratch memory (see include/wush.h).
+namespace wush {
+namespace {
+
+constexpr size_t kStaticScratchFloats = WUSH_STATIC_SCRATCH_BYTES / sizeof(float);
+static __device__ __align__(256) float g_static_partials[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+float* g_static_ptr[kMaxDevices] = {};      // device address of g_static_partials, per device
+
+// Resolves the device address of the array on the CURRENT device (once per device).  In host
+// code the symbol's name is only a handle; kernels need the address the runtime returns.
+cudaError_t static_scratch(float** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_partials);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = static_cast<float*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace wush
+
+extern "C" int wush_calib_moments_static(const void* Xc, int64_t B, int64_t K, int g, float* moments,
+                                         int64_t* count, void* stream) {
+  if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  if (B < 0 || K <= 0 || K % g != 0 || K % 64 != 0 || B > (int64_t)1 << 30 || K > (int64_t)1 << 30)
+    return WUSH_ERR_SHAPE;
+  if (!Xc || !moments || !count) return WUSH_ERR_NULL;
+  if (((reinterpret_cast<uintptr_t>(Xc) | reinterpret_cast<uintptr_t>(moments)) & 15u) != 0) return WUSH_ERR_ALIGN;
+  const size_t per_split = (size_t)K * (size_t)g;                 // floats of one partial set
+  if (per_split > wush::kStaticScratchFloats) return WUSH_ERR_WORKSPACE;   // K * g beyond the built-in scratch
+  if (B == 0) return WUSH_OK;
+  int splits = wush::moments_splits(B, K);
+  const size_t fit = wush::kStaticScratchFloats / per_split;
+  if ((size_t)splits > fit) splits = (int)fit;
+  float* scratch = nullptr;
+  cudaError_t e = wush::static_scratch(&scratch);
+  if (e == cudaSuccess)
+    e = wush::run_calib_moments(Xc, B, K, g, moments, count, scratch, splits, (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : WUSH_ERR_CUDA;
+}

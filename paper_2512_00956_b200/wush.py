@@ -24,8 +24,9 @@ EXPORTS = [
     "wush_status_string", "wush_last_cuda_error", "wush_scale_bytes", "wush_quantize_act",
     "wush_quantize_weight", "wush_quantize_weight_workspace_bytes", "wush_gemm_fp4", "wush_linear",
     "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
-    "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32",
+    "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
 ]
+STATIC_SCRATCH_BYTES = 4 << 20
 
 _lib = None
 
@@ -58,6 +59,8 @@ def lib():
         L.wush_calib_moments.argtypes = [vp, i64, i64, i32, vp, vp, vp, sz, vp]
         L.wush_calib_moments_workspace_bytes.restype = sz
         L.wush_calib_moments_workspace_bytes.argtypes = [i64, i64, i32]
+        L.wush_calib_moments_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]
+        L.wush_calib_moments_static.restype = i32
         L.wush_quantize_f32.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, i32, vp]
         L.wush_transform_act_f32.argtypes = [vp, i64, i64, vp, i32, vp, vp]
         L.wush_transform_weight_f32.argtypes = [vp, i64, i64, vp, i32, vp, vp]
@@ -189,6 +192,20 @@ def calib_moments(Xc, g, moments=None, count=None):
     nws = lib().wush_calib_moments_workspace_bytes(B, K, g)
     ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=Xc.device)
     check(lib().wush_calib_moments(_ptr(Xc), B, K, g, _ptr(moments), _ptr(count), _ptr(ws), ws.numel(), _stream()))
+    return moments, count
+
+
+def calib_moments_static(Xc, g, moments=None, count=None):
+    """wush_calib_moments_static: like calib_moments, but the library's built-in scratch array is
+    used, so no workspace tensor is created here.  For processes that cannot allocate device
+    memory when they call (the outputs are passed in, or made once by the caller)."""
+    _dev(Xc, moments, count)
+    B, K = Xc.shape
+    if moments is None:
+        moments = torch.zeros((K // g, g, g), dtype=torch.float32, device=Xc.device)
+    if count is None:
+        count = torch.zeros(2, dtype=torch.int64, device=Xc.device)
+    check(lib().wush_calib_moments_static(_ptr(Xc), B, K, g, _ptr(moments), _ptr(count), _stream()))
     return moments, count
 
 
