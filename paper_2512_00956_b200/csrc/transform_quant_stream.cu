@@ -1,0 +1,310 @@
+// Streaming variant of the fused block transform + quantise kernel (Eq. 7 inner term) used by
+// the online path: the same arithmetic as transform_quant.cu, restructured so that HBM stays
+// busy.
+//
+//  * Persistent CTAs (one per SM): 1 producer warp + 16 consumer warps.  The producer streams
+//    128-row x 128-channel tiles of X into a 4-stage shared-memory ring with TMA (four
+//    64-byte-wide boxes per tile, no swizzle, no multicast), so up to 96 KB per SM are in flight
+//    without costing a register.
+//  * A work item is (128-channel panel, 128-row block); a CTA takes a contiguous run of items in
+//    panel-major order, so the panel rarely changes.  Each consumer warp owns one 16-row slice
+//    and two of the panel's four 32-channel super-blocks, and keeps the MMA B-fragments of those
+//    two transforms in REGISTERS for as long as the panel stays the same (32 registers): in
+//    steady state the only loads are two 128-bit shared-memory reads per super-block.
+//  * Output permutation: MMA column slot (tile t, n) carries transform row 8*c(n/2) + 2*t + n%2
+//    with c = (0,2,1,3), so after one shuffle with lane^2 every lane owns 8 contiguous code
+//    bytes and a row's 32 bytes leave as one full sector per quad.
+#include <cuda.h>
+
+#include "wush_device.cuh"
+#include "wush_host.h"
+
+namespace wush {
+
+constexpr int SQ_ROWS = 128;
+constexpr int SQ_STAGES = 4;
+constexpr int SQ_CONSUMERS = 16;
+constexpr int SQ_THREADS = (SQ_CONSUMERS + 1) * 32;
+constexpr int SQ_SB_BYTES = SQ_ROWS * 64;              // one super-block of a tile: 128 rows x 64 B
+constexpr int SQ_STAGE_BYTES = 4 * SQ_SB_BYTES;        // 32 KiB
+constexpr int SQ_SMEM = SQ_STAGES * SQ_STAGE_BYTES + 1024 + 128;
+
+__device__ __forceinline__ uint32_t sq_smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ bool sq_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t sq_timer() { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+// bounded wait (about one second); false on expiry or when another role has aborted
+__device__ __forceinline__ bool sq_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < 2048; ++i)
+    if (sq_try_wait(bar, parity)) return true;
+  const uint64_t t0 = sq_timer();
+  while (true) {
+    for (int i = 0; i < 64; ++i)
+      if (sq_try_wait(bar, parity)) return true;
+    if (*abort_flag != 0 || sq_timer() - t0 > 1000000000ull) return false;
+  }
+}
+__device__ __forceinline__ bool sq_elect() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
+template <int G>
+__global__ void __launch_bounds__(SQ_THREADS, 1)
+tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
+                 const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                 int sf_layout, int num_rb, int64_t num_items, int32_t* __restrict__ status) {
+  constexpr int FMT = (G == 32) ? kFmtMX : kFmtNV;
+  extern __shared__ uint8_t sq_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(sq_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SQ_STAGES * SQ_STAGE_BYTES);
+  uint64_t* empty_bar = full_bar + SQ_STAGES;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + SQ_STAGES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < SQ_STAGES; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sq_smem_u32(&full_bar[s])), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sq_smem_u32(&empty_bar[s])), "r"(SQ_CONSUMERS));
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // contiguous run of items for this CTA; item -> (panel, row block), panel-major
+  const int64_t item_begin = (num_items * blockIdx.x) / gridDim.x;
+  const int64_t item_end = (num_items * (blockIdx.x + 1)) / gridDim.x;
+  const int total_sb = (int)(K >> 5);
+
+  if (warp == SQ_CONSUMERS) {
+    // ------------------------------------------------------------------ producer warp
+    int n = 0;
+    for (int64_t it = item_begin; it < item_end; ++it, ++n) {
+      const int s = n % SQ_STAGES;
+      const uint32_t ph = (n / SQ_STAGES) & 1;
+      if (!__all_sync(0xffffffffu, sq_wait(sq_smem_u32(&empty_bar[s]), ph ^ 1, abort_flag))) {
+        if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x40000 | n); *abort_flag = 1; }
+        break;
+      }
+      const int panel = (int)(it / num_rb), rb = (int)(it % num_rb);
+      const int nsb = min(4, total_sb - panel * 4);
+      if (sq_elect()) {
+        const uint32_t bar = sq_smem_u32(&full_bar[s]);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(nsb * SQ_SB_BYTES) : "memory");
+        for (int sb = 0; sb < nsb; ++sb) {
+          const uint32_t dst = sq_smem_u32(smem + s * SQ_STAGE_BYTES + sb * SQ_SB_BYTES);
+          asm volatile(
+              "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+              ::"r"(dst), "l"(&mapX), "r"((panel * 4 + sb) * 32), "r"(rb * SQ_ROWS), "r"(bar) : "memory");
+        }
+      }
+      __syncwarp();
+    }
+    if (*abort_flag != 0) {
+      // a wait expired somewhere: let every tile that was requested land before the CTA exits
+      for (int k = max(0, n - SQ_STAGES); k < n; ++k) {
+        const uint64_t t0 = sq_timer();
+        while (!sq_try_wait(sq_smem_u32(&full_bar[k % SQ_STAGES]), (k / SQ_STAGES) & 1))
+          if (sq_timer() - t0 > 500000000ull) break;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumer warps
+    const int gid = lane >> 2, tig = lane & 3;
+    const int mt = warp & 7;                  // 16-row slice of the tile
+    const int sbp = warp >> 3;                // super-blocks 2*sbp, 2*sbp+1 of the panel
+    const int chunk = ((tig & 1) << 1) | (tig >> 1);          // c(tig) = (0,2,1,3)
+    const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
+    const int64_t KB = K / G;
+    float ts = 1.0f;
+    if (FMT == kFmtNV) ts = *ts_ptr;
+
+    uint4 tf[2][4];                           // B fragments of the two transforms, kept across items
+    int cur_panel = -1;
+    int n = 0;
+    bool ok = true;
+    for (int64_t it = item_begin; it < item_end && ok; ++it, ++n) {
+      const int panel = (int)(it / num_rb), rb = (int)(it % num_rb);
+      const int nsb = min(4, total_sb - panel * 4);
+      if (panel != cur_panel) {
+        cur_panel = panel;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int sb = panel * 4 + 2 * sbp + q;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const int r = 8 * nchunk + 2 * t + (gid & 1);     // transform row for column slot gid of tile t
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (2 * sbp + q < nsb) {
+              if (G == 32) {
+                w = __ldg(reinterpret_cast<const uint4*>(T + ((int64_t)sb * 32 + r) * 32 + 8 * tig));
+              } else if ((r >> 4) == (tig >> 1)) {              // block-diagonal pair: off-diagonal chunks are zero
+                w = __ldg(reinterpret_cast<const uint4*>(T + (((int64_t)sb * 2 + (r >> 4)) * 16 + (r & 15)) * 16 + 8 * (tig & 1)));
+              }
+            }
+            tf[q][t] = w;
+          }
+        }
+      }
+      const int s = n % SQ_STAGES;
+      const uint32_t ph = (n / SQ_STAGES) & 1;
+      if (!__all_sync(0xffffffffu, sq_wait(sq_smem_u32(&full_bar[s]), ph, abort_flag))) {
+        if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x50000 | n); *abort_flag = 1; }
+        ok = false;
+        break;
+      }
+      const uint8_t* tile = smem + s * SQ_STAGE_BYTES;
+      uint4 xa[2], xb[2];
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const uint8_t* p = tile + (2 * sbp + q) * SQ_SB_BYTES + (16 * mt + gid) * 64 + 16 * tig;
+        xa[q] = *reinterpret_cast<const uint4*>(p);
+        xb[q] = *reinterpret_cast<const uint4*>(p + 8 * 64);
+      }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sq_smem_u32(&empty_bar[s])) : "memory");
+
+      if (2 * sbp >= nsb) continue;             // K tail: this warp's super-blocks do not exist
+      const int64_t rA = (int64_t)rb * SQ_ROWS + 16 * mt + gid, rB = rA + 8;
+      const bool okA = rA < M, okB = rB < M;
+      uint32_t wA[2], wB[2], sA[2], sB[2];
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        float acc[4][4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
+          mma_bf16_16816(acc[t], xa[q].x, xb[q].x, xa[q].y, xb[q].y, tf[q][t].x, tf[q][t].y);
+          mma_bf16_16816(acc[t], xa[q].z, xb[q].z, xa[q].w, xb[q].w, tf[q][t].z, tf[q][t].w);
+        }
+        float vA[8], vB[8];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          vA[2 * t] = acc[t][0]; vA[2 * t + 1] = acc[t][1];
+          vB[2 * t] = acc[t][2]; vB[2 * t + 1] = acc[t][3];
+        }
+        float aA = 0.f, aB = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { aA = fmaxf(aA, fabsf(vA[i])); aB = fmaxf(aB, fabsf(vB[i])); }
+        aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 2));       // lanes tig and tig^2 share a g=16 block
+        aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 2));
+        if (G == 32) {
+          aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 1));
+          aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 1));
+        }
+        float mA, mB;
+        if (FMT == kFmtMX) { mx_scale(aA, sA[q], mA); mx_scale(aB, sB[q], mB); }
+        else               { nv_scale(aA, ts, sA[q], mA); nv_scale(aB, ts, sB[q], mB); }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { vA[i] = __fmul_rn(vA[i], mA); vB[i] = __fmul_rn(vB[i], mB); }
+        wA[q] = pack_e2m1x8(vA);
+        wB[q] = pack_e2m1x8(vB);
+      }
+      // ---- codes: lanes 0,1 gather super-block 0, lanes 2,3 super-block 1 (8 contiguous bytes each)
+      {
+        const bool lo = tig < 2;
+        const uint32_t rcvA = __shfl_xor_sync(0xffffffffu, lo ? wA[1] : wA[0], 2);
+        const uint32_t rcvB = __shfl_xor_sync(0xffffffffu, lo ? wB[1] : wB[0], 2);
+        const uint2 oA = lo ? make_uint2(wA[0], rcvA) : make_uint2(rcvA, wA[1]);
+        const uint2 oB = lo ? make_uint2(wB[0], rcvB) : make_uint2(rcvB, wB[1]);
+        const int64_t col = (int64_t)panel * 64 + sbp * 32 + 8 * tig;        // byte column in the code row
+        const bool col_ok = (2 * sbp + (tig >> 1)) < nsb;
+        if (okA && col_ok) *reinterpret_cast<uint2*>(codes + rA * (K >> 1) + col) = oA;
+        if (okB && col_ok) *reinterpret_cast<uint2*>(codes + rB * (K >> 1) + col) = oB;
+      }
+      // ---- scale bytes
+      if (G == 32) {
+        if (tig == 0) {
+          const int64_t kb = (int64_t)panel * 4 + 2 * sbp;
+          if (2 * sbp + 1 < nsb) {
+            if (okA) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rA, kb, KB)) = (uint16_t)(sA[0] | (sA[1] << 8));
+            if (okB) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rB, kb, KB)) = (uint16_t)(sB[0] | (sB[1] << 8));
+          } else {
+            if (okA) scales[sf_offset(sf_layout, rA, kb, KB)] = (uint8_t)sA[0];
+            if (okB) scales[sf_offset(sf_layout, rB, kb, KB)] = (uint8_t)sB[0];
+          }
+        }
+      } else {
+        // lanes tig 0,2 hold the first block of each super-block, lanes 1,3 the second
+        const uint32_t mineA = sA[0] | (sA[1] << 16), mineB = sB[0] | (sB[1] << 16);
+        const uint32_t othA = __shfl_xor_sync(0xffffffffu, mineA, 1), othB = __shfl_xor_sync(0xffffffffu, mineB, 1);
+        if (tig == 0) {
+          const int64_t kb = (int64_t)panel * 8 + 4 * sbp;
+          const uint32_t outA = mineA | (othA << 8), outB = mineB | (othB << 8);
+          if (2 * sbp + 1 < nsb) {
+            if (okA) *reinterpret_cast<uint32_t*>(scales + sf_offset(sf_layout, rA, kb, KB)) = outA;
+            if (okB) *reinterpret_cast<uint32_t*>(scales + sf_offset(sf_layout, rB, kb, KB)) = outB;
+          } else {
+            if (okA) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rA, kb, KB)) = (uint16_t)outA;
+            if (okB) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rB, kb, KB)) = (uint16_t)outB;
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// ------------------------------------------------------------------------------ host side
+typedef CUresult (*SqEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static SqEncodeFn sq_encode_fn() {
+  static SqEncodeFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<SqEncodeFn>(p);
+  }
+  return fn;
+}
+
+// Returns cudaErrorNotSupported when the streaming kernel cannot take the problem (the caller
+// then uses the register-staged kernel).
+cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
+                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, cudaStream_t st) {
+  SqEncodeFn enc = sq_encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  const cuuint32_t box[2] = {32, (cuuint32_t)SQ_ROWS};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorNotSupported;
+  static int sm_count = 0;
+  static bool attr_done = false;
+  cudaError_t e;
+  if (!attr_done) {
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const int num_rb = (int)((M + SQ_ROWS - 1) / SQ_ROWS);
+  const int64_t panels = (K / 32 + 3) / 4;
+  const int64_t items = panels * num_rb;
+  const int grid = (int)(items < sm_count ? items : sm_count);
+  const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
+  if (g == 32)
+    tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, items, status);
+  else
+    tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, items, status);
+  return cudaGetLastError();
+}
+
+}  // namespace wush

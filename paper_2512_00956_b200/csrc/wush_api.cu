@@ -79,7 +79,7 @@ int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T, wush_f
   if (!X || !T || !codes || !scales || (fmt == WUSH_NVFP4 && !x_tensor_scale)) return WUSH_ERR_NULL;
   if (!aligned16(X) || !aligned16(T) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
   if (M == 0) return WUSH_OK;
-  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, (cudaStream_t)stream);
+  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, nullptr, (cudaStream_t)stream);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
@@ -117,7 +117,7 @@ int wush_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const
   if (!device_is_sm100()) return WUSH_ERR_DEVICE;
   const char* why = nullptr;
   cudaError_t e = wush::run_gemm_fp4(Xq, Xs, Wq, Ws, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
-                                     ydt == WUSH_OUT_BF16, status, (cudaStream_t)stream, &why);
+                                     ydt == WUSH_OUT_BF16, status, true, (cudaStream_t)stream, &why);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e, why);
 }
 
@@ -144,10 +144,19 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_
   if (!X || !T || !Wcodes || !Wscales || !Y) return WUSH_ERR_NULL;
   if (fmt == WUSH_NVFP4 && (!x_tensor_scale || !w_tensor_scale)) return WUSH_ERR_NULL;
   if (!aligned16(Wcodes) || !aligned16(Wscales) || !aligned16(Y)) return WUSH_ERR_ALIGN;
-  rc = wush_quantize_act(X, M, K, T, fmt, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, stream);
-  if (rc) return rc;
-  return wush_gemm_fp4(xq, xs, Wcodes, Wscales, M, N, K, fmt, g, x_tensor_scale, w_tensor_scale, Y, ydt, status,
-                       stream);
+  if (!X || !T) return WUSH_ERR_NULL;
+  if (!aligned16(X) || !aligned16(T)) return WUSH_ERR_ALIGN;
+  if (M == 0) return WUSH_OK;
+  if (!device_is_sm100()) return WUSH_ERR_DEVICE;
+  // one status word for both kernels: cleared here, set by whichever bounded wait expires first
+  cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int32_t), (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, status, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const char* why = nullptr;
+  e = wush::run_gemm_fp4(xq, xs, Wcodes, Wscales, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
+                         ydt == WUSH_OUT_BF16, status, false, (cudaStream_t)stream, &why);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e, why);
 }
 
 size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g) {

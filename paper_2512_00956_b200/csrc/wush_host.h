@@ -7,7 +7,10 @@
 namespace wush {
 
 cudaError_t run_quantize_act(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
-                             uint8_t* codes, uint8_t* scales, int sf, cudaStream_t st);
+                             uint8_t* codes, uint8_t* scales, int sf, int32_t* status, cudaStream_t st);
+// streaming (TMA-fed, persistent) variant; cudaErrorNotSupported = problem not covered, use the other kernel
+cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
+                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, cudaStream_t st);
 cudaError_t run_transform_f32(const void* X, int64_t M, int64_t K, const void* T, int g, bool t_is_f32,
                               float* V, cudaStream_t st);
 cudaError_t run_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv, int g,
@@ -24,6 +27,6 @@ cudaError_t run_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float
 // receives a static description when the failure is not a CUDA error (e.g. no driver symbol).
 cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws,
                          int64_t M, int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw,
-                         void* Y, int out_bf16, int32_t* status, cudaStream_t st, const char** why);
+                         void* Y, int out_bf16, int32_t* status, bool clear_status, cudaStream_t st, const char** why);
 
 }  // namespace wush
