@@ -3,9 +3,9 @@
 // busy.
 //
 //  * Persistent CTAs (one per SM): 1 producer warp + 16 consumer warps.  The producer streams
-//    128-row x 128-channel tiles of X into a 4-stage shared-memory ring with TMA (four
-//    64-byte-wide boxes per tile, no swizzle, no multicast), so up to 96 KB per SM are in flight
-//    without costing a register.
+//    128-row x 128-channel tiles of X into a 4-stage shared-memory ring with TMA (two
+//    128-byte-wide boxes per tile, 128-byte swizzle, no multicast), so up to 96 KB per SM are in
+//    flight without costing a register.
 //  * A work item is (128-channel panel, 128-row block); a CTA takes a contiguous run of items in
 //    panel-major order, so the panel rarely changes.  Each consumer warp owns one 16-row slice
 //    and two of the panel's four 32-channel super-blocks, and keeps the MMA B-fragments of those
@@ -58,7 +58,7 @@ template <int G>
 __global__ void __launch_bounds__(SQ_THREADS, 1)
 tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
                  const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
-                 int sf_layout, int num_rb, int64_t num_items, int32_t* __restrict__ status) {
+                 int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status) {
   constexpr int FMT = (G == 32) ? kFmtMX : kFmtNV;
   extern __shared__ uint8_t sq_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(sq_raw) + 1023) & ~uintptr_t(1023));
@@ -78,33 +78,35 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
   __syncthreads();
 
   // contiguous run of items for this CTA; item -> (panel, row block), panel-major
-  const int64_t item_begin = (num_items * blockIdx.x) / gridDim.x;
-  const int64_t item_end = (num_items * (blockIdx.x + 1)) / gridDim.x;
+  const int item_begin = (int)(((int64_t)num_items * blockIdx.x) / gridDim.x);
+  const int item_end = (int)(((int64_t)num_items * (blockIdx.x + 1)) / gridDim.x);
   const int total_sb = (int)(K >> 5);
 
   if (warp == SQ_CONSUMERS) {
     // ------------------------------------------------------------------ producer warp
     int n = 0;
-    for (int64_t it = item_begin; it < item_end; ++it, ++n) {
+    int panel = item_begin / num_rb, rb = item_begin % num_rb;
+    for (int it = item_begin; it < item_end; ++it, ++n) {
       const int s = n % SQ_STAGES;
       const uint32_t ph = (n / SQ_STAGES) & 1;
       if (!__all_sync(0xffffffffu, sq_wait(sq_smem_u32(&empty_bar[s]), ph ^ 1, abort_flag))) {
         if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x40000 | n); *abort_flag = 1; }
         break;
       }
-      const int panel = (int)(it / num_rb), rb = (int)(it % num_rb);
       const int nsb = min(4, total_sb - panel * 4);
       if (sq_elect()) {
         const uint32_t bar = sq_smem_u32(&full_bar[s]);
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(nsb * SQ_SB_BYTES) : "memory");
-        for (int sb = 0; sb < nsb; ++sb) {
-          const uint32_t dst = sq_smem_u32(smem + s * SQ_STAGE_BYTES + sb * SQ_SB_BYTES);
+        const int nbox = nsb >> 1;                       // 64-channel (128-byte) boxes; K % 64 == 0
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(nbox * 2 * SQ_SB_BYTES) : "memory");
+        for (int bx = 0; bx < nbox; ++bx) {
+          const uint32_t dst = sq_smem_u32(smem + s * SQ_STAGE_BYTES + bx * 2 * SQ_SB_BYTES);
           asm volatile(
               "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-              ::"r"(dst), "l"(&mapX), "r"((panel * 4 + sb) * 32), "r"(rb * SQ_ROWS), "r"(bar) : "memory");
+              ::"r"(dst), "l"(&mapX), "r"((panel * 2 + bx) * 64), "r"(rb * SQ_ROWS), "r"(bar) : "memory");
         }
       }
       __syncwarp();
+      if (++rb == num_rb) { rb = 0; ++panel; }
     }
     if (*abort_flag != 0) {
       // a wait expired somewhere: let every tile that was requested land before the CTA exits
@@ -118,8 +120,10 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     // ------------------------------------------------------------------ consumer warps
     const int gid = lane >> 2, tig = lane & 3;
     const int mt = warp & 7;                  // 16-row slice of the tile
+    // MMA row slot gid reads tile row 16*mt + pi(gid), pi = (0,4,1,5,2,6,3,7): the two rows of a
+    // quarter-warp then differ in bit 2, which the swizzle turns into disjoint bank halves
+    const int prow = 16 * mt + ((gid & 1) << 2) + (gid >> 1);
     const int sbp = warp >> 3;                // super-blocks 2*sbp, 2*sbp+1 of the panel
-    const int chunk = ((tig & 1) << 1) | (tig >> 1);          // c(tig) = (0,2,1,3)
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
     float ts = 1.0f;
@@ -128,9 +132,11 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     uint4 tf[2][4];                           // B fragments of the two transforms, kept across items
     int cur_panel = -1;
     int n = 0;
-    bool ok = true;
-    for (int64_t it = item_begin; it < item_end && ok; ++it, ++n) {
-      const int panel = (int)(it / num_rb), rb = (int)(it % num_rb);
+    int panel = item_begin / num_rb, rb = item_begin % num_rb;
+    const int KB32 = (int)KB;
+    const int ktiles = (KB32 + 3) >> 2;
+    const int64_t code_pitch = K >> 1;
+    for (int it = item_begin; it < item_end; ++it, ++n) {
       const int nsb = min(4, total_sb - panel * 4);
       if (panel != cur_panel) {
         cur_panel = panel;
@@ -156,22 +162,25 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
       const uint32_t ph = (n / SQ_STAGES) & 1;
       if (!__all_sync(0xffffffffu, sq_wait(sq_smem_u32(&full_bar[s]), ph, abort_flag))) {
         if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x50000 | n); *abort_flag = 1; }
-        ok = false;
         break;
       }
       const uint8_t* tile = smem + s * SQ_STAGE_BYTES;
       uint4 xa[2], xb[2];
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
-        const uint8_t* p = tile + (2 * sbp + q) * SQ_SB_BYTES + (16 * mt + gid) * 64 + 16 * tig;
+        // box sbp holds this warp's two super-blocks: rows of 128 bytes, 16-byte chunk index XORed
+        // with (row & 7) by the TMA swizzle; rows prow and prow + 8 share the same XOR term
+        const uint8_t* p = tile + sbp * (2 * SQ_SB_BYTES) + prow * 128 + (((4 * q + tig) ^ (prow & 7)) << 4);
         xa[q] = *reinterpret_cast<const uint4*>(p);
-        xb[q] = *reinterpret_cast<const uint4*>(p + 8 * 64);
+        xb[q] = *reinterpret_cast<const uint4*>(p + 8 * 128);
       }
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sq_smem_u32(&empty_bar[s])) : "memory");
 
+      const int this_panel = panel, this_rb = rb;
+      if (++rb == num_rb) { rb = 0; ++panel; }
       if (2 * sbp >= nsb) continue;             // K tail: this warp's super-blocks do not exist
-      const int64_t rA = (int64_t)rb * SQ_ROWS + 16 * mt + gid, rB = rA + 8;
+      const int rA = this_rb * SQ_ROWS + prow, rB = rA + 8;
       const bool okA = rA < M, okB = rB < M;
       uint32_t wA[2], wB[2], sA[2], sB[2];
 #pragma unroll
@@ -179,8 +188,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         float acc[4][4];
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
-          mma_bf16_16816(acc[t], xa[q].x, xb[q].x, xa[q].y, xb[q].y, tf[q][t].x, tf[q][t].y);
+          mma_bf16_16816_first(acc[t], xa[q].x, xb[q].x, xa[q].y, xb[q].y, tf[q][t].x, tf[q][t].y);
           mma_bf16_16816(acc[t], xa[q].z, xb[q].z, xa[q].w, xb[q].w, tf[q][t].z, tf[q][t].w);
         }
         float vA[8], vB[8];
@@ -199,12 +207,23 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
           aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 1));
         }
         float mA, mB;
-        if (FMT == kFmtMX) { mx_scale(aA, sA[q], mA); mx_scale(aB, sB[q], mB); }
-        else               { nv_scale(aA, ts, sA[q], mA); nv_scale(aB, ts, sB[q], mB); }
+        if (FMT == kFmtMX) {
+          mx_scale(aA, sA[q], mA); mx_scale(aB, sB[q], mB);
+        } else {
+          // four distinct scales per quad (row A/B x block 0/1): lane tig computes the one of
+          // (row tig>>1, its own block) and fetches the other row's from lane tig^2
+          const bool mine_is_b = (tig >> 1) != 0;
+          uint32_t sm; float mm;
+          nv_scale(mine_is_b ? aB : aA, ts, sm, mm);
+          const uint32_t so = __shfl_xor_sync(0xffffffffu, sm, 2);
+          const float mo = __shfl_xor_sync(0xffffffffu, mm, 2);
+          sA[q] = mine_is_b ? so : sm; mA = mine_is_b ? mo : mm;
+          sB[q] = mine_is_b ? sm : so; mB = mine_is_b ? mm : mo;
+        }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { vA[i] = __fmul_rn(vA[i], mA); vB[i] = __fmul_rn(vB[i], mB); }
-        wA[q] = pack_e2m1x8(vA);
-        wB[q] = pack_e2m1x8(vB);
+        for (int i = 0; i < 8; i += 2) { mul2_rn(vA[i], vA[i + 1], mA); mul2_rn(vB[i], vB[i + 1], mB); }
+        wA[q] = pack_e2m1x8_fast(vA);
+        wB[q] = pack_e2m1x8_fast(vB);
       }
       // ---- codes: lanes 0,1 gather super-block 0, lanes 2,3 super-block 1 (8 contiguous bytes each)
       {
@@ -213,36 +232,51 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         const uint32_t rcvB = __shfl_xor_sync(0xffffffffu, lo ? wB[1] : wB[0], 2);
         const uint2 oA = lo ? make_uint2(wA[0], rcvA) : make_uint2(rcvA, wA[1]);
         const uint2 oB = lo ? make_uint2(wB[0], rcvB) : make_uint2(rcvB, wB[1]);
-        const int64_t col = (int64_t)panel * 64 + sbp * 32 + 8 * tig;        // byte column in the code row
         const bool col_ok = (2 * sbp + (tig >> 1)) < nsb;
-        if (okA && col_ok) *reinterpret_cast<uint2*>(codes + rA * (K >> 1) + col) = oA;
-        if (okB && col_ok) *reinterpret_cast<uint2*>(codes + rB * (K >> 1) + col) = oB;
+        uint8_t* pa = codes + (int64_t)rA * code_pitch + (this_panel * 64 + sbp * 32 + 8 * tig);
+        if (okA && col_ok) *reinterpret_cast<uint2*>(pa) = oA;
+        if (okB && col_ok) *reinterpret_cast<uint2*>(pa + 8 * code_pitch) = oB;
       }
-      // ---- scale bytes
-      if (G == 32) {
-        if (tig == 0) {
-          const int64_t kb = (int64_t)panel * 4 + 2 * sbp;
-          if (2 * sbp + 1 < nsb) {
-            if (okA) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rA, kb, KB)) = (uint16_t)(sA[0] | (sA[1] << 8));
-            if (okB) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rB, kb, KB)) = (uint16_t)(sB[0] | (sB[1] << 8));
+      // ---- scale bytes: one 16-bit (g=32) or 32-bit (g=16) store per row by lane tig == 0
+      if (tig == 0) {
+        const int kb = (G == 32) ? this_panel * 4 + 2 * sbp : this_panel * 8 + 4 * sbp;
+        int64_t offA, offB;
+        if (sf_layout == 0) {
+          offA = (int64_t)rA * KB32 + kb;
+          offB = offA + 8 * (int64_t)KB32;
+        } else {
+          // rows rA and rA + 8 lie in the same 32-row group of the same 128-row tile
+          offA = ((int64_t)(rA >> 7) * ktiles + (kb >> 2)) * 512 + (rA & 31) * 16 + ((rA & 127) >> 5) * 4 + (kb & 3);
+          offB = offA + 8 * 16;
+        }
+        const bool pair_ok = 2 * sbp + 1 < nsb;
+        if (G == 32) {
+          const uint32_t outA = sA[0] | (sA[1] << 8), outB = sB[0] | (sB[1] << 8);
+          if (pair_ok) {
+            if (okA) *reinterpret_cast<uint16_t*>(scales + offA) = (uint16_t)outA;
+            if (okB) *reinterpret_cast<uint16_t*>(scales + offB) = (uint16_t)outB;
           } else {
-            if (okA) scales[sf_offset(sf_layout, rA, kb, KB)] = (uint8_t)sA[0];
-            if (okB) scales[sf_offset(sf_layout, rB, kb, KB)] = (uint8_t)sB[0];
+            if (okA) scales[offA] = (uint8_t)outA;
+            if (okB) scales[offB] = (uint8_t)outB;
           }
         }
-      } else {
+      }
+      if (G == 16) {
         // lanes tig 0,2 hold the first block of each super-block, lanes 1,3 the second
         const uint32_t mineA = sA[0] | (sA[1] << 16), mineB = sB[0] | (sB[1] << 16);
         const uint32_t othA = __shfl_xor_sync(0xffffffffu, mineA, 1), othB = __shfl_xor_sync(0xffffffffu, mineB, 1);
         if (tig == 0) {
-          const int64_t kb = (int64_t)panel * 8 + 4 * sbp;
+          const int kb = this_panel * 8 + 4 * sbp;
+          int64_t offA, offB;
+          if (sf_layout == 0) { offA = (int64_t)rA * KB32 + kb; offB = offA + 8 * (int64_t)KB32; }
+          else { offA = ((int64_t)(rA >> 7) * ktiles + (kb >> 2)) * 512 + (rA & 31) * 16 + ((rA & 127) >> 5) * 4; offB = offA + 8 * 16; }
           const uint32_t outA = mineA | (othA << 8), outB = mineB | (othB << 8);
           if (2 * sbp + 1 < nsb) {
-            if (okA) *reinterpret_cast<uint32_t*>(scales + sf_offset(sf_layout, rA, kb, KB)) = outA;
-            if (okB) *reinterpret_cast<uint32_t*>(scales + sf_offset(sf_layout, rB, kb, KB)) = outB;
+            if (okA) *reinterpret_cast<uint32_t*>(scales + offA) = outA;
+            if (okB) *reinterpret_cast<uint32_t*>(scales + offB) = outB;
           } else {
-            if (okA) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rA, kb, KB)) = (uint16_t)outA;
-            if (okB) *reinterpret_cast<uint16_t*>(scales + sf_offset(sf_layout, rB, kb, KB)) = (uint16_t)outB;
+            if (okA) *reinterpret_cast<uint16_t*>(scales + offA) = (uint16_t)outA;
+            if (okB) *reinterpret_cast<uint16_t*>(scales + offB) = (uint16_t)outB;
           }
         }
       }
@@ -278,10 +312,10 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   CUtensorMap map;
   const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
   const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  const cuuint32_t box[2] = {32, (cuuint32_t)SQ_ROWS};
+  const cuuint32_t box[2] = {64, (cuuint32_t)SQ_ROWS};
   const cuuint32_t estr[2] = {1, 1};
   if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
-          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorNotSupported;
   static int sm_count = 0;
@@ -298,12 +332,13 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   const int num_rb = (int)((M + SQ_ROWS - 1) / SQ_ROWS);
   const int64_t panels = (K / 32 + 3) / 4;
   const int64_t items = panels * num_rb;
+  if (items > 0x7fffffff || M > 0x7fffff00) return cudaErrorNotSupported;
   const int grid = (int)(items < sm_count ? items : sm_count);
   const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
   if (g == 32)
-    tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, items, status);
+    tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status);
   else
-    tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, items, status);
+    tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status);
   return cudaGetLastError();
 }
 

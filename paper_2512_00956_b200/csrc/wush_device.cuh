@@ -36,6 +36,32 @@ __device__ __forceinline__ uint32_t pack_e2m1x8(const float (&u)[8]) {
   return w;
 }
 
+// Same packing, written so that the four conversions and the byte merge are five instructions:
+// cvt.rn.satfinite.e2m1x2.f32 d, a, b puts a in the high nibble and b in the low one.
+__device__ __forceinline__ uint32_t pack_e2m1x8_fast(const float (&u)[8]) {
+  uint32_t w;
+  asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+      "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+      : "=r"(w)
+      : "f"(u[0]), "f"(u[1]), "f"(u[2]), "f"(u[3]), "f"(u[4]), "f"(u[5]), "f"(u[6]), "f"(u[7]));
+  return w;
+}
+
+// (a, b) * (m, m) with one packed fp32 instruction (round to nearest, no flush)
+__device__ __forceinline__ void mul2_rn(float& a, float& b, float m) {
+  asm("{\n\t.reg .b64 v, s;\n\t"
+      "mov.b64 v, {%0, %1};\n\t"
+      "mov.b64 s, {%2, %2};\n\t"
+      "mul.rn.f32x2 v, v, s;\n\t"
+      "mov.b64 {%0, %1}, v;\n\t}"
+      : "+f"(a), "+f"(b)
+      : "f"(m));
+}
+
 // ---- MXFP4 scale: e = clamp(floor(log2 amax) - 2, -127, 127); returns the E8M0 byte and
 // the exact fp32 multiplier 2^-e.  amax is finite and non-negative.
 __device__ __forceinline__ void mx_scale(float amax, uint32_t& byte, float& mult) {
@@ -67,6 +93,16 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
       "{%0,%1,%2,%3};\n"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// D = A * B (no accumulator input: the zero operand costs no register moves)
+__device__ __forceinline__ void mma_bf16_16816_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                     uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%10,%10,%10,%10};\n"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
 }
 
 // transpose an 8x8 matrix of 16-bit elements held one 32-bit register per lane
