@@ -374,15 +374,19 @@ static bool make_operand_map(CUtensorMap* map, const void* base, int64_t rows, i
 cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws,
                          int64_t M, int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw,
                          void* Y, int out_bf16, int32_t* status, bool clear_status, cudaStream_t st, const char** why) {
-  CUtensorMap mapA, mapB;
-  if (!make_operand_map(&mapA, Xq, M, K / 2, BM) || !make_operand_map(&mapB, Wq, N, K / 2, BN)) {
-    if (why) *why = "cuTensorMapEncodeTiled unavailable or rejected the operand layout";
-    return cudaErrorInvalidValue;
-  }
   cudaError_t e;
   if (status && clear_status) {
     e = cudaMemsetAsync(status, 0, sizeof(int32_t), st);
     if (e != cudaSuccess) return e;
+  }
+  if (M > 128) {
+    e = run_gemm_fp4_2cta(Xq, Xs, Wq, Ws, M, N, K, fmt, tsx, tsw, Y, out_bf16, status, st);
+    if (e != cudaErrorNotSupported) return e;
+  }
+  CUtensorMap mapA, mapB;
+  if (!make_operand_map(&mapA, Xq, M, K / 2, BM) || !make_operand_map(&mapB, Wq, N, K / 2, BN)) {
+    if (why) *why = "cuTensorMapEncodeTiled unavailable or rejected the operand layout";
+    return cudaErrorInvalidValue;
   }
   dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
   if (fmt == kFmtMX) {

@@ -1,0 +1,414 @@
+// Block-scaled FP4 GEMM, two-CTA form (Eq. 7, outer sum) - the kernel wush_gemm_fp4 uses for
+// M > 128.  Same arithmetic as gemm_fp4.cu; different machine mapping:
+//
+//  * Persistent clusters of two CTAs (one cluster per SM pair) walk the 256 x 256 output tiles.
+//    CTA r of a pair owns rows [128 r, 128 r + 128) of the tile: it loads its 128 rows of A and
+//    ITS HALF (128 rows) of the B tile.  tcgen05.mma.cta_group::2 (M = 256, N = 256, K = 64)
+//    reads each CTA's B half from that CTA's shared memory, so every SM streams only half of B
+//    - a single SM cannot feed its tensor cores at the FP4 rate from its own shared memory -
+//    and no TMA multicast is involved anywhere.
+//  * All operand and scale loads are TMA tile loads in the cta_group::2 form, which lets both
+//    CTAs signal the LEADER's "full" mbarrier; the leader's elected MMA thread copies the scale
+//    tiles to tensor memory (tcgen05.cp.cta_group::2 acts on both CTAs), issues the MMAs, and
+//    releases a stage in both CTAs with one multicast tcgen05.commit.
+//  * Eight epilogue warps per CTA drain the 128 x 256 fp32 accumulator (tcgen05.ld), signal the
+//    leader as soon as the last column has been read, and finish their global stores while the
+//    next tile's MMAs already run.  The producers never stop, so the ring is full when they do.
+//
+// Every mbarrier wait is bounded (about two seconds).  On expiry the role records a diagnostic
+// word in *status, raises its CTA's abort flag and falls through to the common exit; the peer
+// CTA's own bounded waits expire in turn, so the closing cluster barrier is always reached.
+#include <cuda.h>
+
+#include "wush_device.cuh"
+#include "wush_host.h"
+
+namespace wush {
+namespace g2 {
+
+constexpr int BM = 256, BN = 256;       // cluster tile
+constexpr int BKB = 128;                // packed-FP4 bytes per row per stage (256 elements)
+constexpr int STAGES = 5;
+constexpr int A_BYTES = 128 * BKB;      // this CTA's 128 rows of A
+constexpr int B_BYTES = 128 * BKB;      // this CTA's 128 rows (half) of B
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = (2 + EPI_WARPS) * 32;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t SFA_COL = 256, SFB_COL = 288;
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;   // clears the CTA-rank bit of a shared::cluster address: rank 0 of the pair
+
+__host__ __device__ constexpr int tps(int fmt) { return fmt == kFmtMX ? 2 : 4; }
+__host__ __device__ constexpr int sf_bytes(int fmt) { return 3 * tps(fmt) * 512; }
+__host__ __device__ constexpr int stage_bytes(int fmt) { return A_BYTES + B_BYTES + sf_bytes(fmt); }
+__host__ __device__ constexpr int smem_bytes(int fmt) { return 1024 + STAGES * stage_bytes(fmt) + 256; }
+
+__device__ __forceinline__ uint32_t s32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t timer_ns() { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < 4096; ++i)
+    if (try_wait(bar, parity)) return true;
+  const uint64_t t0 = timer_ns();
+  while (true) {
+    for (int i = 0; i < 64; ++i)
+      if (try_wait(bar, parity)) return true;
+    if (*abort_flag != 0 || timer_ns() - t0 > 2000000000ull) return false;
+  }
+}
+__device__ __forceinline__ bool elect() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+// TMA tile load whose completion bytes are counted on the pair leader's mbarrier (no multicast)
+__device__ __forceinline__ void tma_2sm(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t leader_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
+}
+__device__ __forceinline__ void commit_both(uint32_t bar) {      // arrives on `bar` in both CTAs of the pair
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void arrive_leader(uint32_t bar) {    // one arrival on the leader's copy of `bar`
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_MASK) : "memory");
+}
+__device__ __forceinline__ void cp_sf2(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+template <int FMT>
+__device__ __forceinline__ void mma2(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t acc) {
+  if (FMT == kFmtMX) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(sfa), "r"(sfb) : "memory");
+  } else {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(sfa), "r"(sfb) : "memory");
+  }
+}
+__device__ __forceinline__ void ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ uint64_t op_desc(uint32_t a) {      // K-major, 128-byte swizzle, 8-row groups 1024 B apart
+  return static_cast<uint64_t>((a & 0x3FFFFu) >> 4) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint64_t sf_desc(uint32_t a) {      // 32 rows x 16 B, no swizzle
+  return static_cast<uint64_t>((a & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(128 >> 4) << 32) | (1ull << 46);
+}
+__device__ __forceinline__ uint32_t idesc2(int fmt, uint32_t sf_byte) {   // M = 256 across the pair, N = 256
+  return (sf_byte << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+         ((fmt == kFmtMX ? 1u : 0u) << 23) | (static_cast<uint32_t>(BM >> 4) << 24) | (sf_byte << 29);
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+
+template <int FMT>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                     const __grid_constant__ CUtensorMap mapSFA, const __grid_constant__ CUtensorMap mapSFB,
+                     int M, int N, int K, const float* __restrict__ tsx, const float* __restrict__ tsw,
+                     void* __restrict__ Yout, int out_bf16, int32_t* __restrict__ status) {
+  constexpr int TPS = tps(FMT);
+  constexpr int KSTEPS_PER_TILE = (FMT == kFmtMX) ? 2 : 1;
+  extern __shared__ uint8_t raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = smem;
+  uint8_t* sB = sA + STAGES * A_BYTES;
+  uint8_t* sSF = sB + STAGES * B_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sSF + STAGES * sf_bytes(FMT));
+  uint64_t* full_bar = bars;                      // used in the leader only
+  uint64_t* empty_bar = bars + STAGES;            // one copy per CTA, released together by the multicast commit
+  uint64_t* tmem_full = bars + 2 * STAGES;        // per CTA
+  uint64_t* tmem_empty = bars + 2 * STAGES + 1;   // leader only: 2 x EPI_WARPS arrivals per tile
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();            // 0 = leader
+  const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+  const int tiles_n = (N + BN - 1) / BN, tiles_m = (M + BM - 1) / BM;
+  const int num_tiles = tiles_m * tiles_n;
+  const int num_kb = (K + 2 * BKB - 1) / (2 * BKB);
+  const int sf_cols = K / (FMT == kFmtMX ? 32 : 16);
+  const int ktiles_total = (sf_cols + 3) >> 2;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(&full_bar[s])), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(&empty_bar[s])), "r"(1));
+    }
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(tmem_full)), "r"(1));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(tmem_empty)), "r"(2 * EPI_WARPS));
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync();                                  // both CTAs' barriers exist before anything remote touches them
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer (one per CTA)
+    int g = 0;                                     // running k-block count across tiles
+    bool ok = true;
+    for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+      const int m0 = (tile / tiles_n) * BM + (int)rank * 128;
+      const int n0 = (tile % tiles_n) * BN;
+      for (int kb = 0; kb < num_kb; ++kb, ++g) {
+        const int s = g % STAGES;
+        const uint32_t ph = (g / STAGES) & 1;
+        if (!__all_sync(0xffffffffu, wait(s32(&empty_bar[s]), ph ^ 1, abort_flag))) {
+          if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x110000 | (rank << 15) | (g & 0x7fff)); *abort_flag = 1; }
+          ok = false;
+          break;
+        }
+        if (elect()) {
+          const uint32_t bar = s32(&full_bar[s]) & PEER_MASK;        // the leader's barrier
+          if (rank == 0)
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(&full_bar[s])), "r"(2 * stage_bytes(FMT)) : "memory");
+          uint8_t* sf = sSF + s * sf_bytes(FMT);
+          tma_2sm(s32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
+          tma_2sm(s32(sB + s * B_BYTES), &mapB, kb * BKB, n0 + (int)rank * 128, bar);
+          tma_2sm(s32(sf), &mapSFA, 0, (m0 >> 7) * ktiles_total + kb * TPS, bar);
+          tma_2sm(s32(sf + TPS * 512), &mapSFB, 0, (n0 >> 7) * ktiles_total + kb * TPS, bar);
+          tma_2sm(s32(sf + 2 * TPS * 512), &mapSFB, 0, ((n0 >> 7) + 1) * ktiles_total + kb * TPS, bar);
+        }
+        __syncwarp();
+      }
+    }
+    if (!ok) {                                     // give copies already in flight time to land before the CTA exits
+      const uint64_t t0 = timer_ns();
+      while (timer_ns() - t0 < 200000ull) { }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (rank == 0) {
+      int g = 0, it = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++it) {
+        if (it > 0) {                               // the epilogues of both CTAs have drained the accumulator
+          if (!__all_sync(0xffffffffu, wait(s32(tmem_empty), (it - 1) & 1, abort_flag))) {
+            if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x130000 | (it & 0xffff)); *abort_flag = 1; }
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % STAGES;
+          const uint32_t ph = (g / STAGES) & 1;
+          if (!__all_sync(0xffffffffu, wait(s32(&full_bar[s]), ph, abort_flag))) {
+            if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x120000 | (g & 0xffff)); *abort_flag = 1; }
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const int tiles = min(TPS, ktiles_total - kb * TPS);
+          const uint32_t sf = s32(sSF + s * sf_bytes(FMT));
+          const int ksteps = min(4, (K - kb * 2 * BKB) / 64);
+          const uint64_t adesc = op_desc(s32(sA + s * A_BYTES));
+          const uint64_t bdesc = op_desc(s32(sB + s * B_BYTES));
+          if (elect()) {
+            for (int i = 0; i < tiles; ++i) {
+              cp_sf2(tmem_base + SFA_COL + 4 * i, sf_desc(sf + i * 512));
+              cp_sf2(tmem_base + SFB_COL + 8 * i, sf_desc(sf + (TPS + i) * 512));
+              cp_sf2(tmem_base + SFB_COL + 8 * i + 4, sf_desc(sf + (2 * TPS + i) * 512));
+            }
+            for (int j = 0; j < ksteps; ++j) {
+              const int t4 = j / KSTEPS_PER_TILE;
+              const uint32_t sfb = (FMT == kFmtMX) ? 2u * (j % KSTEPS_PER_TILE) : 0u;
+              mma2<FMT>(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc2(FMT, sfb), tmem_base + SFA_COL + 4 * t4,
+                        tmem_base + SFB_COL + 8 * t4, (kb | j) != 0);
+            }
+            commit_both(s32(&empty_bar[s]));
+          }
+          __syncwarp();
+        }
+        if (!ok) break;
+        if (elect()) commit_both(s32(tmem_full));
+        __syncwarp();
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (8 warps per CTA)
+    const int q = warp & 3;                        // tensor-memory lane quarter this warp may read
+    const int half = (warp - 2) >> 2;              // columns [128 half, 128 half + 128)
+    float alpha = 1.0f;
+    if (FMT == kFmtNV) alpha = __fmul_rn(*tsx, *tsw);
+    int it = 0;
+    bool ok = true;
+    for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++it) {
+      const int m0 = (tile / tiles_n) * BM + (int)rank * 128;
+      const int n0 = (tile % tiles_n) * BN + half * 128;
+      const int row = m0 + q * 32 + lane;
+      if (!__all_sync(0xffffffffu, wait(s32(tmem_full), it & 1, abort_flag))) {
+        if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x140000 | (rank << 15) | (it & 0x7fff)); *abort_flag = 1; }
+        ok = false;
+        break;
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        const int col = n0 + c * 32;
+        uint32_t r[32];
+        ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 128 + c * 32, r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (c == 3) {
+          // every column of this warp's slice is in registers: hand the accumulator back
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) arrive_leader(s32(tmem_empty));
+        }
+        if (row < M && col < N) {
+          if (out_bf16) {
+            __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(Yout) + (int64_t)row * N + col;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              if (col + 8 * v < N) {
+                uint32_t p[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * e]) * alpha,
+                                                           __uint_as_float(r[8 * v + 2 * e + 1]) * alpha);
+                  p[e] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                *reinterpret_cast<uint4*>(y + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
+              }
+            }
+          } else {
+            float* y = reinterpret_cast<float*>(Yout) + (int64_t)row * N + col;
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              if (col + 4 * v < N)
+                *reinterpret_cast<float4*>(y + 4 * v) =
+                    make_float4(__uint_as_float(r[4 * v]) * alpha, __uint_as_float(r[4 * v + 1]) * alpha,
+                                __uint_as_float(r[4 * v + 2]) * alpha, __uint_as_float(r[4 * v + 3]) * alpha);
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---- common exit: nobody leaves while the peer may still touch this CTA's memory or barriers
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace g2
+
+// ------------------------------------------------------------------------------ host side
+typedef CUresult (*EncFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                          const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                          CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncFn enc_fn() {
+  static EncFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncFn>(p);
+  }
+  return fn;
+}
+static bool map_bytes(CUtensorMap* map, const void* base, int64_t rows, int64_t row_bytes, int box_rows) {
+  const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+  const cuuint32_t box[2] = {(cuuint32_t)g2::BKB, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc_fn()(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// scale buffer as [tiles][128 x int32]: one row per 512-byte scale tile, box = `tiles_per_box` tiles
+static bool map_scales(CUtensorMap* map, const void* base, int64_t total_tiles, int tiles_per_box) {
+  const cuuint64_t dims[2] = {128, (cuuint64_t)total_tiles};
+  const cuuint64_t strides[1] = {512};
+  const cuuint32_t box[2] = {128, (cuuint32_t)tiles_per_box};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc_fn()(map, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int FMT>
+static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& sa, const CUtensorMap& sb,
+                               int M, int N, int K, const float* tsx, const float* tsw, void* Y, int out_bf16,
+                               int32_t* status, cudaStream_t st) {
+  static int clusters = 0;
+  cudaError_t e;
+  if (clusters == 0) {
+    e = cudaFuncSetAttribute(g2::gemm_fp4_2cta_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, g2::smem_bytes(FMT));
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sms & ~1, 1, 1);
+    cfg.blockDim = dim3(g2::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = g2::smem_bytes(FMT);
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, g2::gemm_fp4_2cta_kernel<FMT>, &cfg);
+    if (e != cudaSuccess || n <= 0) { (void)cudaGetLastError(); n = sms / 2; }
+    clusters = n < sms / 2 ? n : sms / 2;
+  }
+  const int tiles = ((M + g2::BM - 1) / g2::BM) * ((N + g2::BN - 1) / g2::BN);
+  const int nc = tiles < clusters ? tiles : clusters;
+  g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, Y,
+                                                                                   out_bf16, status);
+  return cudaGetLastError();
+}
+
+// cudaErrorNotSupported: the caller should use the single-CTA kernel.
+cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws, int64_t M,
+                              int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw, void* Y,
+                              int out_bf16, int32_t* status, cudaStream_t st) {
+  if (!enc_fn()) return cudaErrorNotSupported;
+  const int64_t ktiles = ((K / (fmt == kFmtMX ? 32 : 16)) + 3) / 4;
+  CUtensorMap a, b, sa, sb;
+  if (!map_bytes(&a, Xq, M, K / 2, 128) || !map_bytes(&b, Wq, N, K / 2, 128) ||
+      !map_scales(&sa, Xs, ((M + 127) / 128) * ktiles, g2::tps(fmt)) ||
+      !map_scales(&sb, Ws, ((N + 127) / 128) * ktiles, g2::tps(fmt)))
+    return cudaErrorNotSupported;
+  if (fmt == kFmtMX) return launch_2cta<kFmtMX>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, st);
+  return launch_2cta<kFmtNV>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, st);
+}
+
+}  // namespace wush
