@@ -290,16 +290,21 @@ def run_ours(args):
 
     # ---- rooflines.  Dominant kernel: the FP4 GEMM (dense contraction -> tensor peak for FP4 =
     # measured bf16 burst peak x nominal FP4:bf16 ratio 4).  Quantiser: HBM.
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            traffic = json.load(f)
+    except Exception:
+        traffic = {}
     fp4_peak = peaks["bf16_tflops"] * 4.0
     gemm_tf = flops / (g_ms * 1e-3) / 1e12
     q_bytes = 2.0 * M * K + M * K / 2.0 + M * K / g + 2.0 * K * g
     q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
-    roof = {"bound": "tensor", "kernel": "gemm_fp4_kernel", "achieved": gemm_tf, "peak": fp4_peak, "unit": "TFLOP/s",
-            "frac": gemm_tf / fp4_peak, "traffic": None, "ms": g_ms,
+    roof = {"bound": "tensor", "kernel": "gemm_fp4_2cta_kernel" if M > 128 else "gemm_fp4_kernel", "achieved": gemm_tf, "peak": fp4_peak, "unit": "TFLOP/s",
+            "frac": gemm_tf / fp4_peak, "traffic": traffic.get(f"gemm_fp4_2cta_kernel/config{cfg.index}"), "ms": g_ms,
             "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TF/s x 4 (nominal FP4:bf16)",
             "frac_of_spec_9pf": gemm_tf / 9000.0}
-    roof_q = {"bound": "hbm", "kernel": "transform_quant_kernel", "achieved": q_gbs, "peak": peaks["hbm_gbs"],
-              "unit": "GB/s", "frac": q_gbs / peaks["hbm_gbs"], "traffic": None, "ms": q_ms,
+    roof_q = {"bound": "hbm", "kernel": "tq_stream_kernel", "achieved": q_gbs, "peak": peaks["hbm_gbs"],
+              "unit": "GB/s", "frac": q_gbs / peaks["hbm_gbs"], "traffic": traffic.get(f"tq_stream_kernel/config{cfg.index}"), "ms": q_ms,
               "algorithmic_bytes": q_bytes, "peak_source": peaks["source"], "frac_of_spec_8tbs": q_gbs / 8000.0}
 
     cpu = None
