@@ -290,9 +290,13 @@ def run_ours(args):
 
     # ---- rooflines.  Dominant kernel: the FP4 GEMM (dense contraction -> tensor peak for FP4 =
     # measured bf16 burst peak x nominal FP4:bf16 ratio 4).  Quantiser: HBM.
+    traffic = {}
     try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
-            traffic = json.load(f)
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for ln in f:
+                if ln.strip() and not ln.startswith("#"):
+                    k_, v_ = ln.split()
+                    traffic[k_] = float(v_)
     except Exception:
         traffic = {}
     fp4_peak = peaks["bf16_tflops"] * 4.0
