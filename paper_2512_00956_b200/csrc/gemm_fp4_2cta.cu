@@ -274,18 +274,20 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
         break;
       }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll 1
+      // Read this warp's whole 32-lane x 128-column slice into registers first and hand the accumulator
+      // back at once: the row-scattered global stores below are slow (one sector per lane and
+      // instruction) and must not hold up the next tile's MMAs.
+      uint32_t r[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 128 + c * 32, r[c]);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) arrive_leader(s32(tmem_empty));
+#pragma unroll
       for (int c = 0; c < 4; ++c) {
         const int col = n0 + c * 32;
-        uint32_t r[32];
-        ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 128 + c * 32, r);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (c == 3) {
-          // every column of this warp's slice is in registers: hand the accumulator back
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) arrive_leader(s32(tmem_empty));
-        }
         if (row < M && col < N) {
           if (out_bf16) {
             __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(Yout) + (int64_t)row * N + col;
@@ -295,8 +297,8 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
                 uint32_t p[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                  __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * e]) * alpha,
-                                                           __uint_as_float(r[8 * v + 2 * e + 1]) * alpha);
+                  __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[c][8 * v + 2 * e]) * alpha,
+                                                           __uint_as_float(r[c][8 * v + 2 * e + 1]) * alpha);
                   p[e] = *reinterpret_cast<uint32_t*>(&h);
                 }
                 *reinterpret_cast<uint4*>(y + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
@@ -308,8 +310,8 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
             for (int v = 0; v < 8; ++v) {
               if (col + 4 * v < N)
                 *reinterpret_cast<float4*>(y + 4 * v) =
-                    make_float4(__uint_as_float(r[4 * v]) * alpha, __uint_as_float(r[4 * v + 1]) * alpha,
-                                __uint_as_float(r[4 * v + 2]) * alpha, __uint_as_float(r[4 * v + 3]) * alpha);
+                    make_float4(__uint_as_float(r[c][4 * v]) * alpha, __uint_as_float(r[c][4 * v + 1]) * alpha,
+                                __uint_as_float(r[c][4 * v + 2]) * alpha, __uint_as_float(r[c][4 * v + 3]) * alpha);
             }
           }
         }
