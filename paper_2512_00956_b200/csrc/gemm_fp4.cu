@@ -373,14 +373,15 @@ static bool make_operand_map(CUtensorMap* map, const void* base, int64_t rows, i
 
 cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws,
                          int64_t M, int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw,
-                         void* Y, int out_bf16, int32_t* status, bool clear_status, cudaStream_t st, const char** why) {
+                         void* Y, int out_bf16, int32_t* status, bool clear_status, bool after_quantizer, cudaStream_t st,
+                         const char** why) {
   cudaError_t e;
   if (status && clear_status) {
     e = cudaMemsetAsync(status, 0, sizeof(int32_t), st);
     if (e != cudaSuccess) return e;
   }
   if (M > 128) {
-    e = run_gemm_fp4_2cta(Xq, Xs, Wq, Ws, M, N, K, fmt, tsx, tsw, Y, out_bf16, status, st);
+    e = run_gemm_fp4_2cta(Xq, Xs, Wq, Ws, M, N, K, fmt, tsx, tsw, Y, out_bf16, status, after_quantizer, st);
     if (e != cudaErrorNotSupported) return e;
   }
   CUtensorMap mapA, mapB;

@@ -186,6 +186,9 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     // ------------------------------------------------------------------ producer (one per CTA)
     int g = 0;                                     // running k-block count across tiles
     bool ok = true;
+    // Launched as a programmatic dependent of the quantiser (wush_linear), everything above overlapped with
+    // that kernel's tail; its output may be read only after this point.  A no-op for a plain launch.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
       const int m0 = (tile / tiles_n) * BM + (int)rank * 128;
       const int n0 = (tile % tiles_n) * BN;
@@ -377,7 +380,7 @@ static bool map_scales(CUtensorMap* map, const void* base, int64_t total_tiles, 
 template <int FMT>
 static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& sa, const CUtensorMap& sb,
                                int M, int N, int K, const float* tsx, const float* tsw, void* Y, int out_bf16,
-                               int32_t* status, cudaStream_t st) {
+                               int32_t* status, bool pdl, cudaStream_t st) {
   static int clusters = 0;
   cudaError_t e;
   if (clusters == 0) {
@@ -401,15 +404,29 @@ static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const
   }
   const int tiles = ((M + g2::BM - 1) / g2::BM) * ((N + g2::BN - 1) / g2::BN);
   const int nc = tiles < clusters ? tiles : clusters;
-  g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, Y,
-                                                                                   out_bf16, status);
-  return cudaGetLastError();
+  if (!pdl) {
+    g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, Y,
+                                                                                     out_bf16, status);
+    return cudaGetLastError();
+  }
+  // programmatic dependent launch: this grid may start while the preceding kernel of the stream drains
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * nc, 1, 1);
+  cfg.blockDim = dim3(g2::THREADS, 1, 1);
+  cfg.dynamicSmemBytes = g2::smem_bytes(FMT);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, g2::gemm_fp4_2cta_kernel<FMT>, a, b, sa, sb, M, N, K, tsx, tsw, Y, out_bf16, status);
 }
 
 // cudaErrorNotSupported: the caller should use the single-CTA kernel.
 cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws, int64_t M,
                               int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw, void* Y,
-                              int out_bf16, int32_t* status, cudaStream_t st) {
+                              int out_bf16, int32_t* status, bool pdl, cudaStream_t st) {
   if (!enc_fn()) return cudaErrorNotSupported;
   const int64_t ktiles = ((K / (fmt == kFmtMX ? 32 : 16)) + 3) / 4;
   CUtensorMap a, b, sa, sb;
@@ -417,8 +434,8 @@ cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_
       !map_scales(&sa, Xs, ((M + 127) / 128) * ktiles, g2::tps(fmt)) ||
       !map_scales(&sb, Ws, ((N + 127) / 128) * ktiles, g2::tps(fmt)))
     return cudaErrorNotSupported;
-  if (fmt == kFmtMX) return launch_2cta<kFmtMX>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, st);
-  return launch_2cta<kFmtNV>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, st);
+  if (fmt == kFmtMX) return launch_2cta<kFmtMX>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, pdl, st);
+  return launch_2cta<kFmtNV>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, pdl, st);
 }
 
 }  // namespace wush

@@ -76,6 +76,9 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // let a programmatic dependent (the GEMM of wush_linear) be scheduled as SMs free up; it still waits
+  // for this whole grid before reading the codes
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // contiguous run of items for this CTA; item -> (panel, row block), panel-major
   const int item_begin = (int)(((int64_t)num_items * blockIdx.x) / gridDim.x);

@@ -117,7 +117,7 @@ int wush_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const
   if (!device_is_sm100()) return WUSH_ERR_DEVICE;
   const char* why = nullptr;
   cudaError_t e = wush::run_gemm_fp4(Xq, Xs, Wq, Ws, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
-                                     ydt == WUSH_OUT_BF16, status, true, (cudaStream_t)stream, &why);
+                                     ydt == WUSH_OUT_BF16, status, true, false, (cudaStream_t)stream, &why);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e, why);
 }
 
@@ -155,7 +155,7 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_
   if (e != cudaSuccess) return cuda_fail(e);
   const char* why = nullptr;
   e = wush::run_gemm_fp4(xq, xs, Wcodes, Wscales, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
-                         ydt == WUSH_OUT_BF16, status, false, (cudaStream_t)stream, &why);
+                         ydt == WUSH_OUT_BF16, status, false, true, (cudaStream_t)stream, &why);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e, why);
 }
 

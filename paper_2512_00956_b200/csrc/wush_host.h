@@ -27,11 +27,12 @@ cudaError_t run_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float
 // receives a static description when the failure is not a CUDA error (e.g. no driver symbol).
 cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws,
                          int64_t M, int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw,
-                         void* Y, int out_bf16, int32_t* status, bool clear_status, cudaStream_t st, const char** why);
+                         void* Y, int out_bf16, int32_t* status, bool clear_status, bool after_quantizer, cudaStream_t st,
+                         const char** why);
 
 // two-CTA persistent variant (M > 128); cudaErrorNotSupported = use the single-CTA kernel
 cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws, int64_t M,
                               int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw, void* Y,
-                              int out_bf16, int32_t* status, cudaStream_t st);
+                              int out_bf16, int32_t* status, bool pdl, cudaStream_t st);
 
 }  // namespace wush
