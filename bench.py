@@ -165,7 +165,7 @@ def run_ours(args):
 
     Xh_bits = synth.activations(cfg, M=M)
     W, Xc = up(synth.weights(cfg)), up(synth.calibration(cfg))
-    layer = prepare.QuantizedLinear(W, Xc, fmt)
+    layer = prepare.QuantizedLinear(W, Xc, fmt, transform=args.transform)
     X0 = up(Xh_bits)
     ws_bytes = wush.linear_workspace_bytes(M, K, g)
     stream = torch.cuda.current_stream()
@@ -338,7 +338,7 @@ def run_ours(args):
     line = {"metric": METRIC, "value": rate / 1e12, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": t_max * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
-            "config": {"workload": cfg.name, "M": M, "K": K, "N": N, "format": fmt, "g": g, "y_dtype": args.out,
+            "config": {"workload": cfg.name, "M": M, "K": K, "N": N, "format": fmt, "g": g, "y_dtype": args.out, "transform": args.transform,
                        "l2": f"cold data: {nsets} rotating buffer sets of {set_bytes / 1e6:.0f} MB (> 2x L2)",
                        "launch": "one CUDA graph of K steps" if used_graph else "eager loop", "tokens_per_rank": M},
             "roofline": roof, "roofline_quant": roof_q,
@@ -362,6 +362,8 @@ def main():
     ap.add_argument("--fmt", default=None, choices=[None, "mxfp4", "nvfp4"])
     ap.add_argument("--m", type=int, default=None, help="override the token count (config 5 sweep)")
     ap.add_argument("--out", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--transform", default="wush", choices=["wush", "hadamard", "identity"],
+                    help="activation-side transform: per-block WUSH (default), one shared Hadamard, or none")
     ap.add_argument("--ref-rows", type=int, default=2048, help="token rows in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -53,16 +53,35 @@ def build_transforms(mom_w, n_w, mom_x, n_x, lam=0.01):
     return T_bf16.contiguous(), Tinv.to(torch.float32).contiguous()
 
 
+def fixed_transforms(kind, C, d, device):
+    """The data-independent comparison transforms of Sec. 5 / Table 1, in the layout the kernels take:
+    "hadamard" (the same normalised Hadamard matrix for every block, the H + Quant baseline) or
+    "identity" (None + Quant).  Returns (T bf16 [C,d,d], Tinv fp32 [C,d,d]) with Tinv = T^-T of the
+    stored bf16 values, exactly as for WUSH."""
+    if kind == "hadamard":
+        T1 = hadamard(d, device)
+    elif kind == "identity":
+        T1 = torch.eye(d, dtype=torch.float64, device=device)
+    else:
+        raise ValueError(kind)
+    T_bf16 = T1.to(torch.bfloat16)
+    Tinv = torch.linalg.inv(T_bf16.to(torch.float64)).transpose(0, 1).to(torch.float32)
+    return T_bf16.expand(C, d, d).contiguous(), Tinv.expand(C, d, d).contiguous()
+
+
 class QuantizedLinear:
     """Holds what the online call needs: T, packed W~ codes, TILED scale bytes, tensor scales."""
 
-    def __init__(self, W, Xc, fmt, lam=0.01):
+    def __init__(self, W, Xc, fmt, lam=0.01, transform="wush"):
         f, g = wush.FORMATS[fmt]
         self.fmt, self.g = fmt, g
         self.N, self.K = W.shape
-        mom_w, cnt_w = wush.calib_moments(W, g)
-        mom_x, cnt_x = wush.calib_moments(Xc, g)
-        self.T, self.Tinv = build_transforms(mom_w, int(cnt_w[0].item()), mom_x, int(cnt_x[0].item()), lam)
+        if transform == "wush":
+            mom_w, cnt_w = wush.calib_moments(W, g)
+            mom_x, cnt_x = wush.calib_moments(Xc, g)
+            self.T, self.Tinv = build_transforms(mom_w, int(cnt_w[0].item()), mom_x, int(cnt_x[0].item()), lam)
+        else:
+            self.T, self.Tinv = fixed_transforms(transform, self.K // g, g, W.device)
         self.w_codes, self.w_scales, self.w_tensor_scale = wush.quantize_weight(W, self.Tinv, fmt, sf=wush.SF_TILED)
         if fmt == "nvfp4":
             v = wush.transform_act_f32(Xc, self.T, g)                            # static activation tensor scale

@@ -243,3 +243,27 @@ def test_linear_bf16_output_config2_bench_configuration():
     assert wush.linear_status(wsp, X.shape[0], X.shape[1], 16) == 0
     Yo = F.round_to_bf16(L.forward(d["X"]))
     assert rel_fro(Y.float().cpu().numpy(), Yo) <= 1e-3
+
+
+@pytest.mark.parametrize("kind", ["hadamard", "identity"])
+def test_fixed_transform_variants_run_through_the_same_kernels(kind):
+    """H + Quant and None + Quant (Sec. 5) are the WUSH kernels with a replicated / identity T; on a layer
+    with outlier channels the ordering of Table 1 must show: WUSH < Hadamard < identity (MXFP4)."""
+    from paper_2512_00956_b200 import prepare
+    cfg = synth.CONFIGS[1]
+    d = synth.layer_inputs(cfg, M=128, N=256, K=512, B=512)
+    W, Xc, X = dev_bf16(d["W"]), dev_bf16(d["Xc"]), dev_bf16(d["X"])
+    Y0 = F.bf16_bits_to_f64(d["X"]) @ F.bf16_bits_to_f64(d["W"]).T
+    loss = {}
+    for k in ("wush", kind):
+        layer = prepare.QuantizedLinear(W, Xc, "mxfp4", transform=k)
+        loss[k] = rel_fro(layer(X).cpu().numpy(), Y0)
+    assert loss["wush"] < loss[kind]
+    # and the fixed transform agrees with the oracle run on the same transform bytes
+    layer = prepare.QuantizedLinear(W, Xc, "mxfp4", transform=kind)
+    T = layer.T.double().cpu().numpy()
+    Tx = layer.Tinv.double().cpu().numpy()
+    v32 = P.transform_blocks(F.bf16_bits_to_f64(d["X"]), T).astype(np.float32)
+    w32 = P.transform_blocks(F.bf16_bits_to_f64(d["W"]), Tx).astype(np.float32)
+    Yo = P.dequantized_product(Q.dequantize(*Q.quantize(v32, "mxfp4"), "mxfp4"), Q.dequantize(*Q.quantize(w32, "mxfp4"), "mxfp4"))
+    assert rel_fro(layer(X).cpu().numpy(), Yo) <= 1e-3
