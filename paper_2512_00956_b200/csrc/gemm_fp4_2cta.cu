@@ -32,9 +32,11 @@ constexpr int STAGES = 5;
 constexpr int A_BYTES = 128 * BKB;      // this CTA's 128 rows of A
 constexpr int B_BYTES = 128 * BKB;      // this CTA's 128 rows (half) of B
 constexpr int EPI_WARPS = 8;
-constexpr int THREADS = (2 + EPI_WARPS) * 32;
+constexpr int SF_WARP = 2 + EPI_WARPS;     // copies scale tiles to tensor memory (leader CTA)
+constexpr int THREADS = (3 + EPI_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t SFA_COL = 256, SFB_COL = 288;
+// scale tiles: one 48-column buffer per ring stage (A scales 16 columns, B scales 32), after the accumulator
+constexpr uint32_t SF_COL0 = 256, SF_STRIDE = 48, SFB_OFF = 16;
 constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;   // clears the CTA-rank bit of a shared::cluster address: rank 0 of the pair
 
 __host__ __device__ constexpr int tps(int fmt) { return fmt == kFmtMX ? 2 : 4; }
@@ -82,6 +84,10 @@ __device__ __forceinline__ void tma_2sm(uint32_t dst, const CUtensorMap* map, in
 __device__ __forceinline__ void commit_both(uint32_t bar) {      // arrives on `bar` in both CTAs of the pair
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void commit_leader(uint32_t bar) {    // arrives on the leader's `bar` only
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)1) : "memory");
 }
 __device__ __forceinline__ void arrive_leader(uint32_t bar) {    // one arrival on the leader's copy of `bar`
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_MASK) : "memory");
@@ -150,7 +156,8 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   uint64_t* empty_bar = bars + STAGES;            // one copy per CTA, released together by the multicast commit
   uint64_t* tmem_full = bars + 2 * STAGES;        // per CTA
   uint64_t* tmem_empty = bars + 2 * STAGES + 1;   // leader only: 2 x EPI_WARPS arrivals per tile
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
+  uint64_t* sf_full = bars + 2 * STAGES + 2;      // leader only: scale tiles of a stage are in tensor memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * STAGES + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -166,6 +173,7 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     for (int s = 0; s < STAGES; ++s) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(&full_bar[s])), "r"(1));
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(&empty_bar[s])), "r"(1));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(&sf_full[s])), "r"(1));
     }
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(tmem_full)), "r"(1));
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(tmem_empty)), "r"(2 * EPI_WARPS));
@@ -235,28 +243,22 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
           const int s = g % STAGES;
           const uint32_t ph = (g / STAGES) & 1;
-          if (!__all_sync(0xffffffffu, wait(s32(&full_bar[s]), ph, abort_flag))) {
+          // the scale warp has seen this stage's operands land and has copied its scale tiles to tensor memory
+          if (!__all_sync(0xffffffffu, wait(s32(&sf_full[s]), ph, abort_flag))) {
             if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x120000 | (g & 0xffff)); *abort_flag = 1; }
             ok = false;
             break;
           }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const int tiles = min(TPS, ktiles_total - kb * TPS);
-          const uint32_t sf = s32(sSF + s * sf_bytes(FMT));
           const int ksteps = min(4, (K - kb * 2 * BKB) / 64);
           const uint64_t adesc = op_desc(s32(sA + s * A_BYTES));
           const uint64_t bdesc = op_desc(s32(sB + s * B_BYTES));
+          const uint32_t sfa_t = tmem_base + SF_COL0 + SF_STRIDE * s, sfb_t = sfa_t + SFB_OFF;
           if (elect()) {
-            for (int i = 0; i < tiles; ++i) {
-              cp_sf2(tmem_base + SFA_COL + 4 * i, sf_desc(sf + i * 512));
-              cp_sf2(tmem_base + SFB_COL + 8 * i, sf_desc(sf + (TPS + i) * 512));
-              cp_sf2(tmem_base + SFB_COL + 8 * i + 4, sf_desc(sf + (2 * TPS + i) * 512));
-            }
             for (int j = 0; j < ksteps; ++j) {
               const int t4 = j / KSTEPS_PER_TILE;
               const uint32_t sfb = (FMT == kFmtMX) ? 2u * (j % KSTEPS_PER_TILE) : 0u;
-              mma2<FMT>(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc2(FMT, sfb), tmem_base + SFA_COL + 4 * t4,
-                        tmem_base + SFB_COL + 8 * t4, (kb | j) != 0);
+              mma2<FMT>(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc2(FMT, sfb), sfa_t + 4 * t4, sfb_t + 8 * t4, (kb | j) != 0);
             }
             commit_both(s32(&empty_bar[s]));
           }
@@ -267,10 +269,43 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
         __syncwarp();
       }
     }
+  } else if (warp == SF_WARP) {
+    // ------------------------------------------------------------------ scale-tile copier (leader CTA only)
+    // A second issuing thread: tcgen05.cp costs about as many issue cycles per K slab as the MMAs do, so the
+    // copies run from their own warp.  Buffer s of tensor memory belongs to ring stage s: when stage s has
+    // been refilled, the MMAs that read its previous scales have completed (that is what freed the stage).
+    if (rank == 0) {
+      int g = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % STAGES;
+          const uint32_t ph = (g / STAGES) & 1;
+          if (!__all_sync(0xffffffffu, wait(s32(&full_bar[s]), ph, abort_flag))) {
+            if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x150000 | (g & 0xffff)); *abort_flag = 1; }
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const int tiles = min(TPS, ktiles_total - kb * TPS);
+          const uint32_t sf = s32(sSF + s * sf_bytes(FMT));
+          const uint32_t sfa_t = tmem_base + SF_COL0 + SF_STRIDE * s, sfb_t = sfa_t + SFB_OFF;
+          if (elect()) {
+            for (int i = 0; i < tiles; ++i) {
+              cp_sf2(sfa_t + 4 * i, sf_desc(sf + i * 512));
+              cp_sf2(sfb_t + 8 * i, sf_desc(sf + (TPS + i) * 512));
+              cp_sf2(sfb_t + 8 * i + 4, sf_desc(sf + (2 * TPS + i) * 512));
+            }
+            commit_leader(s32(&sf_full[s]));
+          }
+          __syncwarp();
+        }
+      }
+    }
   } else {
     // ------------------------------------------------------------------ epilogue (8 warps per CTA)
     const int q = warp & 3;                        // tensor-memory lane quarter this warp may read
-    const int half = (warp - 2) >> 2;              // columns [128 half, 128 half + 128)
+    const int half = (warp - 2) >> 2;              // columns [128 half, 128 half + 128)  (warps 2..9)
     float alpha = 1.0f;
     if (FMT == kFmtNV) alpha = __fmul_rn(*tsx, *tsw);
     int it = 0;
