@@ -8,9 +8,10 @@
 //    - a single SM cannot feed its tensor cores at the FP4 rate from its own shared memory -
 //    and no TMA multicast is involved anywhere.
 //  * All operand and scale loads are TMA tile loads in the cta_group::2 form, which lets both
-//    CTAs signal the LEADER's "full" mbarrier; the leader's elected MMA thread copies the scale
-//    tiles to tensor memory (tcgen05.cp.cta_group::2 acts on both CTAs), issues the MMAs, and
-//    releases a stage in both CTAs with one multicast tcgen05.commit.
+//    CTAs signal the LEADER's "full" mbarrier.  Two issuing threads work in the leader: one
+//    copies each stage's scale tiles to tensor memory (tcgen05.cp.cta_group::2 acts on both
+//    CTAs; one 48-column buffer per ring stage), the other issues the MMAs and releases the
+//    stage in both CTAs with one multicast tcgen05.commit.
 //  * Eight epilogue warps per CTA drain the 128 x 256 fp32 accumulator (tcgen05.ld), signal the
 //    leader as soon as the last column has been read, and finish their global stores while the
 //    next tile's MMAs already run.  The producers never stop, so the ring is full when they do.
