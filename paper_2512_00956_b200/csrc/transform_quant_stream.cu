@@ -200,9 +200,13 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
           vA[2 * t] = acc[t][0]; vA[2 * t + 1] = acc[t][1];
           vB[2 * t] = acc[t][2]; vB[2 * t + 1] = acc[t][3];
         }
-        float aA = 0.f, aB = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { aA = fmaxf(aA, fabsf(vA[i])); aB = fmaxf(aB, fabsf(vB[i])); }
+        // AbsMax of the lane's 8 values per row as a tree of 3-input maxima (sm_100 has a 3-input FMNMX)
+        float aA = fmaxf(fmaxf(fabsf(vA[0]), fabsf(vA[1])), fabsf(vA[2]));
+        aA = fmaxf(fmaxf(aA, fabsf(vA[3])), fabsf(vA[4]));
+        aA = fmaxf(fmaxf(aA, fabsf(vA[5])), fmaxf(fabsf(vA[6]), fabsf(vA[7])));
+        float aB = fmaxf(fmaxf(fabsf(vB[0]), fabsf(vB[1])), fabsf(vB[2]));
+        aB = fmaxf(fmaxf(aB, fabsf(vB[3])), fabsf(vB[4]));
+        aB = fmaxf(fmaxf(aB, fabsf(vB[5])), fmaxf(fabsf(vB[6]), fabsf(vB[7])));
         aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 2));       // lanes tig and tig^2 share a g=16 block
         aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 2));
         if (G == 32) {
