@@ -3,10 +3,12 @@
 // MXFP4 uses tcgen05.mma kind::mxf4 (E8M0 scales, one per 32 elements); NVFP4 uses
 // kind::mxf4nvf4 (E4M3 scales, one per 16 elements).  Accumulation is fp32 in tensor memory.
 //
-// One CTA computes one 128 x 256 tile of Y.  Warp 0 streams operands: per 256-element K slab
-// two TMA tile loads (128-byte swizzle, K-major packed FP4 bytes) and the matching scale tiles
-// (plain bulk copies of the 512-byte GEMM-native scale tiles) into a 4-stage ring guarded by
-// full/empty mbarriers.  One thread of warp 1 copies the scale tiles into tensor memory
+// This is the kernel for M <= 128 (decode, small batches), where the layer is bound by streaming
+// the weights once from HBM: one CTA computes one 128 x 128 tile of Y, two CTAs share an SM, so
+// N/128 CTAs keep every SM pulling weight bytes.  (M > 128 goes to the two-CTA kernel.)
+// Warp 0 streams operands: per 256-element K slab two TMA tile loads (128-byte swizzle, K-major
+// packed FP4 bytes) and the matching scale tiles (plain bulk copies of the 512-byte GEMM-native
+// scale tiles) into a 3-stage ring guarded by full/empty mbarriers.  One thread of warp 1 copies the scale tiles into tensor memory
 // (tcgen05.cp) and issues four K=64 MMAs per slab; tcgen05.commit releases the stage.
 // Warps 2-5 drain the accumulator (tcgen05.ld), apply alpha and store Y.
 //
@@ -22,18 +24,18 @@
 namespace wush {
 
 constexpr int BM = 128;             // tile rows (tokens)
-constexpr int BN = 256;             // tile columns (output channels)
+constexpr int BN = 128;             // tile columns (output channels)
 constexpr int BKB = 128;            // bytes of packed FP4 per row per stage = 256 elements
-constexpr int STAGES = 4;
+constexpr int STAGES = 3;           // two CTAs share an SM: six stages in flight per SM
 constexpr int A_BYTES = BM * BKB;   // 16 KiB
-constexpr int B_BYTES = BN * BKB;   // 32 KiB
+constexpr int B_BYTES = BN * BKB;   // 16 KiB
 constexpr int GEMM_THREADS = 192;
-constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t SFA_COL = 256;   // tensor-memory column of the A scales (after the 256 accumulator columns)
-constexpr uint32_t SFB_COL = 288;   // B scales: 8 columns per scale tile (two 128-row groups)
+constexpr uint32_t TMEM_COLS = 256;  // two co-resident CTAs fit in the 512 columns of an SM
+constexpr uint32_t SFA_COL = 128;   // tensor-memory column of the A scales (after the 128 accumulator columns)
+constexpr uint32_t SFB_COL = 160;   // B scales: 4 columns per scale tile
 
 __host__ __device__ constexpr int sf_tiles_per_stage(int fmt) { return fmt == kFmtMX ? 2 : 4; }
-__host__ __device__ constexpr int stage_sf_bytes(int fmt) { return 3 * sf_tiles_per_stage(fmt) * 512; }
+__host__ __device__ constexpr int stage_sf_bytes(int fmt) { return 2 * sf_tiles_per_stage(fmt) * 512; }
 __host__ __device__ constexpr int gemm_smem_bytes(int fmt) {
   return 1024 /*alignment slack*/ + STAGES * (A_BYTES + B_BYTES + stage_sf_bytes(fmt)) + 256 /*barriers*/;
 }
@@ -156,18 +158,18 @@ __device__ __forceinline__ uint32_t instr_desc(int fmt, uint32_t sf_byte) {
 
 // ------------------------------------------------------------------------------ the kernel
 template <int FMT>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const uint8_t* __restrict__ SFA, const uint8_t* __restrict__ SFB, int M, int N, int K,
                 const float* __restrict__ tsx, const float* __restrict__ tsw, void* __restrict__ Yout,
-                int out_bf16, int32_t* __restrict__ status) {
+                int out_bf16, int32_t* __restrict__ status, int a_box_bytes) {
   constexpr int TPS = sf_tiles_per_stage(FMT);           // scale tiles (4 scale columns each) per stage
   constexpr int KSTEPS_PER_TILE = (FMT == kFmtMX) ? 2 : 1;  // K=64 MMAs covered by one scale tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = sA + STAGES * A_BYTES;
-  uint8_t* sSF = sB + STAGES * B_BYTES;                   // per stage: [A tiles][B group 0 tiles][B group 1 tiles]
+  uint8_t* sSF = sB + STAGES * B_BYTES;                   // per stage: [A tiles][B tiles]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sSF + STAGES * stage_sf_bytes(FMT));
   uint64_t* full_bar = bars;
   uint64_t* empty_bar = bars + STAGES;
@@ -214,18 +216,17 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         break;
       }
       const int tiles = min(TPS, ktiles_total - kb * TPS);
-      const bool grp1 = (n0 + 128) < ((N + 127) & ~127);      // second 128-row scale group exists
       const uint32_t sf_bytes = tiles * 512;
       const uint32_t bar = smem_u32(&full_bar[s]);
       uint8_t* sf = sSF + s * stage_sf_bytes(FMT);
       if (elect_one()) {
-        mbar_expect_tx(bar, A_BYTES + B_BYTES + sf_bytes * (grp1 ? 3 : 2));
+        // the A box covers only round_up(M, 8) rows when M < 128: the rows of the stage below it keep stale
+        // bytes, which only reach accumulator rows that are never stored
+        mbar_expect_tx(bar, a_box_bytes + B_BYTES + sf_bytes * 2);
         tma_load_2d(smem_u32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
         tma_load_2d(smem_u32(sB + s * B_BYTES), &mapB, kb * BKB, n0, bar);
         bulk_load_1d(smem_u32(sf), SFA + ((int64_t)(m0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
         bulk_load_1d(smem_u32(sf + TPS * 512), SFB + ((int64_t)(n0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
-        if (grp1)
-          bulk_load_1d(smem_u32(sf + 2 * TPS * 512), SFB + ((int64_t)((n0 >> 7) + 1) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
       }
       __syncwarp();
       ++issued;
@@ -261,14 +262,13 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       if (elect_one()) {
         for (int i = 0; i < tiles; ++i) {
           tc_cp_sf(tmem_base + SFA_COL + 4 * i, scale_desc(sf + i * 512));
-          tc_cp_sf(tmem_base + SFB_COL + 8 * i, scale_desc(sf + (TPS + i) * 512));
-          tc_cp_sf(tmem_base + SFB_COL + 8 * i + 4, scale_desc(sf + (2 * TPS + i) * 512));
+          tc_cp_sf(tmem_base + SFB_COL + 4 * i, scale_desc(sf + (TPS + i) * 512));
         }
         for (int j = 0; j < ksteps; ++j) {
           const int tile = j / KSTEPS_PER_TILE;
           const uint32_t sf_byte = (FMT == kFmtMX) ? 2u * (j % KSTEPS_PER_TILE) : 0u;
           tc_mma<FMT>(tmem_base, adesc + 2 * j, bdesc + 2 * j, instr_desc(FMT, sf_byte),
-                      tmem_base + SFA_COL + 4 * tile, tmem_base + SFB_COL + 8 * tile, (kb | j) != 0);
+                      tmem_base + SFA_COL + 4 * tile, tmem_base + SFB_COL + 4 * tile, (kb | j) != 0);
         }
         tc_commit(smem_u32(&empty_bar[s]));
       }
@@ -385,7 +385,8 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
     if (e != cudaErrorNotSupported) return e;
   }
   CUtensorMap mapA, mapB;
-  if (!make_operand_map(&mapA, Xq, M, K / 2, BM) || !make_operand_map(&mapB, Wq, N, K / 2, BN)) {
+  const int a_rows = M >= BM ? BM : (int)((M + 7) / 8 * 8);
+  if (!make_operand_map(&mapA, Xq, M, K / 2, a_rows) || !make_operand_map(&mapB, Wq, N, K / 2, BN)) {
     if (why) *why = "cuTensorMapEncodeTiled unavailable or rejected the operand layout";
     return cudaErrorInvalidValue;
   }
@@ -398,7 +399,7 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
       attr_done = true;
     }
     gemm_fp4_kernel<kFmtMX><<<grid, GEMM_THREADS, gemm_smem_bytes(kFmtMX), st>>>(
-        mapA, mapB, Xs, Ws, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status);
+        mapA, mapB, Xs, Ws, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, a_rows * BKB);
   } else {
     static bool attr_done = false;
     if (!attr_done) {
@@ -407,7 +408,7 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
       attr_done = true;
     }
     gemm_fp4_kernel<kFmtNV><<<grid, GEMM_THREADS, gemm_smem_bytes(kFmtNV), st>>>(
-        mapA, mapB, Xs, Ws, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status);
+        mapA, mapB, Xs, Ws, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, a_rows * BKB);
   }
   return cudaGetLastError();
 }
