@@ -144,6 +144,24 @@ int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* momen
                        int64_t* count, void* workspace, size_t workspace_bytes, void* stream);
 size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g);
 
+/* Offline transform construction (Algorithm 1 for every block, and the pairing of Eq. 6):
+ *   from the UNNORMALISED second-moment sums of the weights (mom_w, over rows_w = d_out rows) and of
+ *   the calibration activations (mom_x, over rows_x = d_batch tokens), both fp32 [K/g][g][g] as
+ *   wush_calib_moments produces them, compute per block
+ *       W', X' = lower Cholesky factors of the damped moments  M + lambda * tr(M)/g * I,
+ *       U S V^T = SVD(W'^T X'),   T_wush = H S^-1/2 U^T W'^T   (H: normalised Sylvester-Hadamard),
+ *   T     <- bf16(T_wush)          [K/g][g][g]   (input of wush_quantize_act / wush_linear)
+ *   Tinv  <- (T)^-T in fp32        [K/g][g][g]   (= T_xvsh for the stored T; input of wush_quantize_weight)
+ *   info  optional int32[K/g] on the device: 0 = ok, 1 = a Cholesky pivot was not positive,
+ *         2 = the Jacobi SVD did not converge, 3 = T was singular.  May be NULL.
+ * The SVD is unique only up to signs and the order of equal singular values (Lemma A.1); the
+ * convention here is: singular values descending, each row of U^T W'^T signed so that its
+ * largest-magnitude entry is positive.  fp64 arithmetic throughout.
+ * Errors: NULL / SHAPE (incl. lambda < 0, rows <= 0) / FORMAT / ALIGN / CUDA. */
+int wush_build_transforms(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x,
+                          int64_t K, int g, float lambda, void* T, float* Tinv, int32_t* info,
+                          void* stream);
+
 /* wush_calib_moments without a workspace argument.  (No counterpart in the paper: this is
  * a packaging variant of the call above, added for hosts where this library must not and
  * cannot obtain device memory at call time - for example a serving process whose allocator

@@ -1,0 +1,250 @@
+// Algorithm 1 ("Compute WUSH for One Block") and the inverse-transpose pairing of Eq. 6 on the
+// device: one CTA per block of d = g channels, everything in fp64 in shared memory.
+//
+//   M_W, M_X   <- moment sums / row counts, symmetrised, damped:  M + lambda * tr(M)/d * I
+//   W', X'     <- lower Cholesky factors
+//   U S V^T    <- SVD of W'^T X', by one-sided Jacobi on (W'^T X')^T = X'^T W' (its right singular
+//                 vectors are U); round-robin pair ordering, d/2 independent rotations per step
+//   T_wush     <- H S^-1/2 U^T W'^T   (singular values descending; each row of U^T W'^T signed so that its
+//                 largest-magnitude entry is positive - Lemma A.1's factor-independent quantity)
+//   T_hat      <- bf16(T_wush)                      (what the online kernel multiplies activations with)
+//   T_xvsh     <- (T_hat)^-T in fp64, stored as fp32 (what the offline weight path uses)
+//
+// This is offline glue between the calibration-moment kernel and the weight quantiser: O(d^3) per
+// block, a few hundred blocks per layer.  info[c] != 0 flags a block whose factorisation failed
+// (1: non-positive Cholesky pivot, 2: Jacobi did not converge, 3: singular transform).
+#include "../../include/wush.h"
+#include "wush_device.cuh"
+#include "wush_host.h"
+
+namespace wush {
+
+constexpr int BT_THREADS = 128;
+
+template <int D>
+__device__ void cholesky_lower(double* A, int* fail) {       // in place; upper triangle zeroed
+  for (int j = 0; j < D; ++j) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double s = A[j * D + j];
+      for (int k = 0; k < j; ++k) s -= A[j * D + k] * A[j * D + k];
+      if (!(s > 0.0)) { *fail = 1; s = 1.0; }
+      A[j * D + j] = sqrt(s);
+    }
+    __syncthreads();
+    const double piv = A[j * D + j];
+    for (int i = j + 1 + threadIdx.x; i < D; i += BT_THREADS) {
+      double s = A[i * D + j];
+      for (int k = 0; k < j; ++k) s -= A[i * D + k] * A[j * D + k];
+      A[i * D + j] = s / piv;
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < D * D; idx += BT_THREADS)
+    if ((idx % D) > (idx / D)) A[idx] = 0.0;
+  __syncthreads();
+}
+
+template <int D>
+__global__ void __launch_bounds__(BT_THREADS)
+build_transforms_kernel(const float* __restrict__ mom_w, double inv_nw, const float* __restrict__ mom_x, double inv_nx,
+                        double lambda, __nv_bfloat16* __restrict__ T_out, float* __restrict__ Tinv_out,
+                        int32_t* __restrict__ info) {
+  extern __shared__ double sm[];
+  double* Wp = sm;                 // M_W -> W'
+  double* Xp = Wp + D * D;         // M_X -> X'
+  double* Bm = Xp + D * D;         // X'^T W', columns orthogonalised by Jacobi
+  double* Jm = Bm + D * D;         // accumulated rotations = U
+  double* Rm = Jm + D * D;         // U^T W'^T (sorted, signed), later the inverse work matrix
+  double* Tm = Rm + D * D;         // T_wush / T_hat
+  __shared__ double sigma[D];
+  __shared__ double red[2];
+  __shared__ int perm[D];
+  __shared__ int fail, rotated;
+  const int c = blockIdx.x, tid = threadIdx.x;
+  const float* mw = mom_w + (size_t)c * D * D;
+  const float* mx = mom_x + (size_t)c * D * D;
+  if (tid == 0) { fail = 0; red[0] = red[1] = 0.0; }
+  __syncthreads();
+
+  // ---- moments: normalise, symmetrise, damp
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+    const int i = idx / D, j = idx % D;
+    Wp[idx] = 0.5 * ((double)mw[i * D + j] + (double)mw[j * D + i]) * inv_nw;
+    Xp[idx] = 0.5 * ((double)mx[i * D + j] + (double)mx[j * D + i]) * inv_nx;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double tw = 0.0, tx = 0.0;
+    for (int i = 0; i < D; ++i) { tw += Wp[i * D + i]; tx += Xp[i * D + i]; }
+    red[0] = lambda * tw / D; red[1] = lambda * tx / D;
+  }
+  __syncthreads();
+  if (tid < D) { Wp[tid * D + tid] += red[0]; Xp[tid * D + tid] += red[1]; }
+  __syncthreads();
+  cholesky_lower<D>(Wp, &fail);
+  cholesky_lower<D>(Xp, &fail);
+
+  // ---- B = X'^T W'  (= (W'^T X')^T),  J = I
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+    const int i = idx / D, j = idx % D;
+    double s = 0.0;
+    for (int k = 0; k < D; ++k) s += Xp[k * D + i] * Wp[k * D + j];
+    Bm[idx] = s;
+    Jm[idx] = (i == j) ? 1.0 : 0.0;
+  }
+  __syncthreads();
+
+  // ---- one-sided Jacobi: rotate column pairs of B (and J) until all pairs are orthogonal.
+  // Round-robin schedule: D-1 steps per sweep, D/2 disjoint pairs per step; a group of GS threads owns a pair.
+  constexpr int PAIRS = D / 2;
+  constexpr int GS = BT_THREADS / PAIRS;            // 8 (D = 32) or 16 (D = 16) threads per pair
+  const int pair = tid / GS, gl = tid % GS;
+  const unsigned gmask = (GS == 32) ? 0xffffffffu : (((1u << GS) - 1u) << ((tid % 32) / GS * GS));
+  int sweep = 0;
+  for (; sweep < 40; ++sweep) {
+    if (tid == 0) rotated = 0;
+    __syncthreads();
+    for (int step = 0; step < D - 1; ++step) {
+      // circle method: index 0 stays, indices 1..D-1 rotate; slot m meets slot D-1-m
+      const int a = (pair == 0) ? 0 : (pair + step) % (D - 1) + 1;
+      const int b = (pair == 0) ? step % (D - 1) + 1 : (D - 1 - pair + step) % (D - 1) + 1;
+      const int p = min(a, b), q = max(a, b);
+      double al = 0.0, be = 0.0, ga = 0.0;
+      for (int r = gl; r < D; r += GS) {
+        const double x = Bm[r * D + p], y = Bm[r * D + q];
+        al += x * x; be += y * y; ga += x * y;
+      }
+#pragma unroll
+      for (int o = GS / 2; o > 0; o >>= 1) {
+        al += __shfl_xor_sync(gmask, al, o);
+        be += __shfl_xor_sync(gmask, be, o);
+        ga += __shfl_xor_sync(gmask, ga, o);
+      }
+      if (fabs(ga) > 1e-15 * sqrt(al * be) && al > 0.0 && be > 0.0) {
+        const double zeta = (be - al) / (2.0 * ga);
+        const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+        const double cs = 1.0 / sqrt(1.0 + t * t), sn = cs * t;
+        for (int r = gl; r < D; r += GS) {
+          const double x = Bm[r * D + p], y = Bm[r * D + q];
+          Bm[r * D + p] = cs * x - sn * y; Bm[r * D + q] = sn * x + cs * y;
+          const double u = Jm[r * D + p], v = Jm[r * D + q];
+          Jm[r * D + p] = cs * u - sn * v; Jm[r * D + q] = sn * u + cs * v;
+        }
+        if (gl == 0 && fabs(ga) > 1e-13 * sqrt(al * be)) rotated = 1;
+      }
+      __syncthreads();
+    }
+    if (rotated == 0) break;
+    __syncthreads();
+  }
+  if (tid == 0 && sweep >= 40) fail = 2;
+
+  // ---- singular values, descending order
+  if (tid < D) {
+    double s = 0.0;
+    for (int r = 0; r < D; ++r) s += Bm[r * D + tid] * Bm[r * D + tid];
+    sigma[tid] = sqrt(s);
+  }
+  __syncthreads();
+  if (tid < D) {
+    int rank = 0;
+    for (int j = 0; j < D; ++j) rank += (sigma[j] > sigma[tid]) || (sigma[j] == sigma[tid] && j < tid);
+    perm[rank] = tid;
+  }
+  __syncthreads();
+
+  // ---- R = U^T W'^T, rows in sorted order, signed
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+    const int i = idx / D, k = idx % D;
+    const int ci = perm[i];
+    double s = 0.0;
+    for (int m = 0; m < D; ++m) s += Jm[m * D + ci] * Wp[k * D + m];
+    Rm[idx] = s;
+  }
+  __syncthreads();
+  if (tid < D) {
+    int best = 0; double bv = -1.0;
+    for (int k = 0; k < D; ++k) { const double v = fabs(Rm[tid * D + k]); if (v > bv) { bv = v; best = k; } }
+    const double sg = (Rm[tid * D + best] < 0.0) ? -1.0 : 1.0;
+    const double sc = sg / sqrt(sigma[perm[tid]]);
+    for (int k = 0; k < D; ++k) Rm[tid * D + k] *= sc;              // S^-1/2 folded in
+  }
+  __syncthreads();
+
+  // ---- T = H (S^-1/2 R),  H[a][i] = (-1)^popcount(a & i) / sqrt(D);  T_hat = bf16(T)
+  const double hnorm = rsqrt((double)D);
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+    const int a = idx / D, k = idx % D;
+    double s = 0.0;
+    for (int i = 0; i < D; ++i) s += ((__popc(a & i) & 1) ? -Rm[i * D + k] : Rm[i * D + k]);
+    const __nv_bfloat16 tb = __double2bfloat16(s * hnorm);
+    T_out[(size_t)c * D * D + idx] = tb;
+    Tm[idx] = (double)__bfloat162float(tb);
+  }
+  __syncthreads();
+
+  // ---- inverse of T_hat by Gauss-Jordan with partial pivoting (Rm becomes the inverse); T_xvsh = inverse^T
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) Rm[idx] = ((idx / D) == (idx % D)) ? 1.0 : 0.0;
+  __syncthreads();
+  for (int col = 0; col < D; ++col) {
+    if (tid == 0) {
+      int pr = col; double pv = fabs(Tm[col * D + col]);
+      for (int r = col + 1; r < D; ++r) if (fabs(Tm[r * D + col]) > pv) { pv = fabs(Tm[r * D + col]); pr = r; }
+      perm[0] = pr;
+      if (!(pv > 0.0)) fail = 3;
+    }
+    __syncthreads();
+    const int pr = perm[0];
+    if (pr != col) {
+      for (int k = tid; k < D; k += BT_THREADS) {
+        double t = Tm[col * D + k]; Tm[col * D + k] = Tm[pr * D + k]; Tm[pr * D + k] = t;
+        t = Rm[col * D + k]; Rm[col * D + k] = Rm[pr * D + k]; Rm[pr * D + k] = t;
+      }
+    }
+    __syncthreads();
+    const double piv = Tm[col * D + col];
+    __syncthreads();
+    for (int k = tid; k < D; k += BT_THREADS) { Tm[col * D + k] /= piv; Rm[col * D + k] /= piv; }
+    __syncthreads();
+    // eliminate column `col` from every other row; factors are read before any row is modified
+    {
+      double* fac = Bm;                       // reuse: D factors
+      for (int r = tid; r < D; r += BT_THREADS) fac[r] = (r == col) ? 0.0 : Tm[r * D + col];
+      __syncthreads();
+      for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+        const int r = idx / D, k = idx % D;
+        const double f = fac[r];
+        if (f != 0.0) { Tm[idx] -= f * Tm[col * D + k]; Rm[idx] -= f * Rm[col * D + k]; }
+      }
+    }
+    __syncthreads();
+  }
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+    const int j = idx / D, k = idx % D;
+    Tinv_out[(size_t)c * D * D + idx] = (float)Rm[k * D + j];      // transpose of the inverse
+  }
+  if (tid == 0 && info != nullptr) info[c] = fail;
+}
+
+cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* mom_x, int64_t n_x, int64_t K, int g,
+                                 double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st) {
+  const int C = (int)(K / g);
+  const size_t smem = 6 * (size_t)g * g * sizeof(double);
+  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(T);
+  cudaError_t e;
+  if (g == 32) {
+    static bool done = false;
+    if (!done) {
+      e = cudaFuncSetAttribute(build_transforms_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      done = true;
+    }
+    build_transforms_kernel<32><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info);
+  } else {
+    build_transforms_kernel<16><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace wush

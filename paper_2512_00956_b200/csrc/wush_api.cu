@@ -178,6 +178,17 @@ int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* momen
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
+int wush_build_transforms(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x, int64_t K, int g,
+                          float lambda, void* T, float* Tinv, int32_t* info, void* stream) {
+  if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  if (K <= 0 || K % g != 0 || rows_w <= 0 || rows_x <= 0 || !(lambda >= 0.0f)) return WUSH_ERR_SHAPE;
+  if (!mom_w || !mom_x || !T || !Tinv) return WUSH_ERR_NULL;
+  if (!aligned16(mom_w) || !aligned16(mom_x) || !aligned16(T) || !aligned16(Tinv)) return WUSH_ERR_ALIGN;
+  cudaError_t e = wush::run_build_transforms(mom_w, rows_w, mom_x, rows_x, K, g, (double)lambda, T, Tinv, info,
+                                             (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
 int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, int g, const float* tensor_scale,
                       uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf, void* stream) {
   int rc = check_fmt(fmt, g);

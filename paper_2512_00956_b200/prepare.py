@@ -1,10 +1,10 @@
 """Offline preparation of one linear layer (Algorithm 2, RTN case) on the GPU.
 
-Second moments come from the library's calibration kernel (`wush_calib_moments`), the weight
-quantisation from `wush_quantize_weight`.  The d x d factorisations of Algorithm 1 in between
-(damped Cholesky, SVD, H S^-1/2 U^T W'^T and the inverse-transpose of Eq. 6) are O(d^3) per
-block and are batched through torch.linalg in fp64 on the device: they are glue between two
-kernels, not part of the online path.
+Second moments come from the library's calibration kernel (`wush_calib_moments`), the d x d
+factorisations of Algorithm 1 and the inverse-transpose of Eq. 6 from `wush_build_transforms`,
+the weight quantisation from `wush_quantize_weight`: nothing leaves the device.
+`build_transforms` below is the same construction written with torch.linalg; it is kept as an
+independent cross-check of the kernel and is not used by `QuantizedLinear`.
 
 Conventions (the paper leaves them open): damping ratio lambda = 0.01; singular values
 descending and each row of U^T W'^T signed so that its largest-magnitude entry is positive
@@ -79,7 +79,11 @@ class QuantizedLinear:
         if transform == "wush":
             mom_w, cnt_w = wush.calib_moments(W, g)
             mom_x, cnt_x = wush.calib_moments(Xc, g)
-            self.T, self.Tinv = build_transforms(mom_w, int(cnt_w[0].item()), mom_x, int(cnt_x[0].item()), lam)
+            # Algorithm 1 + Eq. 6 for every block in the library's own kernel (fp64 Cholesky, Jacobi SVD)
+            self.T, self.Tinv, self.info = wush.build_transforms(mom_w, int(cnt_w[0].item()), mom_x,
+                                                                 int(cnt_x[0].item()), g, lam)
+            if int(self.info.abs().max().item()) != 0:
+                raise wush.WushError("wush_build_transforms: a block failed to factorise (see info)")
         else:
             self.T, self.Tinv = fixed_transforms(transform, self.K // g, g, W.device)
         self.w_codes, self.w_scales, self.w_tensor_scale = wush.quantize_weight(W, self.Tinv, fmt, sf=wush.SF_TILED)

@@ -25,6 +25,7 @@ EXPORTS = [
     "wush_quantize_weight", "wush_quantize_weight_workspace_bytes", "wush_gemm_fp4", "wush_linear",
     "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
+    "wush_build_transforms",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -59,6 +60,8 @@ def lib():
         L.wush_calib_moments.argtypes = [vp, i64, i64, i32, vp, vp, vp, sz, vp]
         L.wush_calib_moments_workspace_bytes.restype = sz
         L.wush_calib_moments_workspace_bytes.argtypes = [i64, i64, i32]
+        L.wush_build_transforms.argtypes = [vp, i64, vp, i64, i64, i32, ctypes.c_float, vp, vp, vp, vp]
+        L.wush_build_transforms.restype = i32
         L.wush_calib_moments_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]
         L.wush_calib_moments_static.restype = i32
         L.wush_quantize_f32.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, i32, vp]
@@ -193,6 +196,19 @@ def calib_moments(Xc, g, moments=None, count=None):
     ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=Xc.device)
     check(lib().wush_calib_moments(_ptr(Xc), B, K, g, _ptr(moments), _ptr(count), _ptr(ws), ws.numel(), _stream()))
     return moments, count
+
+
+def build_transforms(mom_w, rows_w, mom_x, rows_x, g, lam=0.01):
+    """Moment sums fp32 [K/g,g,g] (+ row counts) -> (T bf16 [K/g,g,g], Tinv fp32 [K/g,g,g], info int32 [K/g])."""
+    _dev(mom_w, mom_x)
+    C = mom_w.shape[0]
+    K = C * g
+    T = torch.empty((C, g, g), dtype=torch.bfloat16, device=mom_w.device)
+    Tinv = torch.empty((C, g, g), dtype=torch.float32, device=mom_w.device)
+    info = torch.zeros(max(C, 4), dtype=torch.int32, device=mom_w.device)
+    check(lib().wush_build_transforms(_ptr(mom_w), int(rows_w), _ptr(mom_x), int(rows_x), K, g, float(lam), _ptr(T),
+                                      _ptr(Tinv), _ptr(info), _stream()))
+    return T, Tinv, info[:C]
 
 
 def calib_moments_static(Xc, g, moments=None, count=None):

@@ -267,3 +267,42 @@ def test_fixed_transform_variants_run_through_the_same_kernels(kind):
     w32 = P.transform_blocks(F.bf16_bits_to_f64(d["W"]), Tx).astype(np.float32)
     Yo = P.dequantized_product(Q.dequantize(*Q.quantize(v32, "mxfp4"), "mxfp4"), Q.dequantize(*Q.quantize(w32, "mxfp4"), "mxfp4"))
     assert rel_fro(layer(X).cpu().numpy(), Yo) <= 1e-3
+
+
+# ------------------------------------------------------------------ Algorithm 1 on the device
+@pytest.mark.parametrize("fmt,K", [("mxfp4", 1024), ("nvfp4", 512)])
+def test_build_transforms_kernel_against_oracle_and_identities(fmt, K):
+    """wush_build_transforms: same conventions as the oracle, so the stored bf16 transforms agree to about
+    one bf16 step; and the identities of Eq. 6 / the equalisation appendix hold on what it returns."""
+    from oracle import wush_transform as WT
+    g = G[fmt]
+    cfg = synth.CONFIGS[1]
+    d = synth.layer_inputs(cfg, M=16, N=768, K=K, B=640)
+    Wv, Xcv = F.bf16_bits_to_f64(d["W"]), F.bf16_bits_to_f64(d["Xc"])
+    sW, sX = P.second_moment_sums(Wv, g), P.second_moment_sums(Xcv, g)
+    T, Tinv, info = wush.build_transforms(dev(sW.astype(np.float32)), Wv.shape[0], dev(sX.astype(np.float32)),
+                                          Xcv.shape[0], g, 0.01)
+    _sync()
+    assert int(info.abs().max().item()) == 0
+    Tg = T.double().cpu().numpy(); Tig = Tinv.double().cpu().numpy()
+    bits, That, Tx = WT.build_transforms(sW / Wv.shape[0], sX / Xcv.shape[0], 0.01)
+    scale = np.abs(That).max(axis=(1, 2), keepdims=True)
+    assert np.all(np.abs(Tg - That) <= 2.0 ** -7 * np.abs(That) + 2e-3 * scale)
+    assert np.mean(Tg == That) > 0.9                                   # most entries round to the same bf16 value
+    C = K // g
+    for c in range(C):
+        assert np.allclose(Tig[c] @ Tg[c].T, np.eye(g), atol=1e-5)      # Eq. 6 on the stored values
+    mX = sX / Xcv.shape[0]
+    for c in range(0, C, 3):                                            # equalised diagonal, up to bf16 rounding of T
+        A = Tg[c] @ WT.damped(mX[c], 0.01) @ Tg[c].T
+        assert np.ptp(np.diag(A)) <= 0.05 * np.diag(A).mean()
+    # and the layer prepared from it reaches the oracle's quantisation-error level
+    L = P.PreparedLayer(d["W"], d["Xc"], fmt)
+    X, W = dev_bf16(d["X"]), dev_bf16(d["W"])
+    wq, ws, tsw = wush.quantize_weight(W, Tinv, fmt, sf=wush.SF_TILED)
+    tsx = dev(np.full(4, L.ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
+    Y, _ = wush.linear(X, T, wq, ws, fmt, tsx, tsw)
+    _sync()
+    Y0 = F.bf16_bits_to_f64(d["X"]) @ Wv.T
+    lg, lo = rel_fro(Y.cpu().numpy(), Y0), rel_fro(L.forward(d["X"]), Y0)
+    assert abs(lg - lo) <= 0.15 * lo, (lg, lo)
