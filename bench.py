@@ -269,29 +269,60 @@ def run_ours(args):
         b_.record(stream)
         torch.cuda.synchronize()
         return a_.elapsed_time(b_) / reps
-    Bc = Xc.shape[0]
-    mom_ms = once(lambda: wush.calib_moments(Xc, g))
-    wq_ms = once(lambda: wush.quantize_weight(W, layer.Tinv, fmt, sf=wush.SF_TILED))
-    offline = {"calib_moments": {"ms": mom_ms, "GB/s": (2.0 * Bc * K + 4.0 * K * g) / (mom_ms * 1e-3) / 1e9, "tokens": Bc},
+    # moments of the weight matrix itself (the larger of the two inputs of Algorithm 2), caller-owned buffers
+    mom_buf = torch.zeros((K // g, g, g), dtype=torch.float32, device=dev)
+    cnt_buf = torch.zeros(2, dtype=torch.int64, device=dev)
+    mom_ws = torch.empty(max(16, wush.lib().wush_calib_moments_workspace_bytes(N, K, g)), dtype=torch.uint8, device=dev)
+    mom_ms = once(lambda: wush.calib_moments(W, g, mom_buf, cnt_buf, mom_ws), reps=10)
+    wq_out = (torch.empty_like(layer.w_codes), torch.empty_like(layer.w_scales),
+              torch.zeros(4, dtype=torch.float32, device=dev), torch.empty(256, dtype=torch.uint8, device=dev))
+    wq_ms = once(lambda: wush.quantize_weight(W, layer.Tinv, fmt, sf=wush.SF_TILED, out=wq_out), reps=10)
+    offline = {"calib_moments": {"ms": mom_ms, "GB/s": (2.0 * N * K + 4.0 * K * g) / (mom_ms * 1e-3) / 1e9, "rows": N,
+                                 "note": "second-moment sums of W[N,K]; warm L2 (same buffers every repetition)"},
                "quantize_weight": {"ms": wq_ms, "GB/s": (2.0 * N * K * (2 if fmt == "nvfp4" else 1) + N * K / 2.0 + N * K / g) / (wq_ms * 1e-3) / 1e9,
-                                   "note": "NVFP4 reads W twice (AbsMax pass + quantise pass); includes torch allocations of the binding"}}
+                                   "note": "NVFP4 reads W twice (AbsMax pass + quantise pass); warm L2"}}
 
     # ---- end to end through the public call with HOST buffers: pinned X in, Y back out, every step
     Xh = torch.from_numpy(Xh_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
-    Yh = torch.empty((M, N), dtype=out_dtype).pin_memory()
-    n_e2e = max(5, min(args.steps, 50))
-    d0 = sets[0]
-    for _ in range(2):
-        d0["X"].copy_(Xh, non_blocking=True); step(d0); Yh.copy_(d0["Y"], non_blocking=True)
+    n_e2e = max(6, min(args.steps, 60))
+    # Three streams: the pinned-host -> device copy of step i+1, the kernels of step i and the device -> host
+    # copy of step i-1 overlap (the copy engines are full duplex); every step still moves its own input in
+    # and its own result out inside the timed region.
+    s_in, s_c, s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+    nb3 = min(3, nsets)
+    ev_in = [torch.cuda.Event() for _ in range(nb3)]
+    ev_c = [torch.cuda.Event() for _ in range(nb3)]
+    ev_out = [torch.cuda.Event() for _ in range(nb3)]
+    Yh3 = [torch.empty((M, N), dtype=out_dtype).pin_memory() for _ in range(nb3)]
+
+    def e2e_loop(n):
+        for i in range(n):
+            b = i % nb3
+            d_ = sets[b]
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_c[b])                 # the kernels that last read this X buffer are done
+                d_["X"].copy_(Xh, non_blocking=True)
+                ev_in[b].record(s_in)
+            with torch.cuda.stream(s_c):
+                s_c.wait_event(ev_in[b])
+                s_c.wait_event(ev_out[b])                # the previous result in this Y buffer has left
+                step(d_)
+                ev_c[b].record(s_c)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_c[b])
+                Yh3[b].copy_(d_["Y"], non_blocking=True)
+                ev_out[b].record(s_out)
+
+    e2e_loop(3)
     torch.cuda.synchronize()
     D.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for i in range(n_e2e):
-        d_ = sets[i % nsets]
-        d_["X"].copy_(Xh, non_blocking=True)
-        step(d_)
-        Yh.copy_(d_["Y"], non_blocking=True)
+    for st_ in (s_in, s_c, s_out):
+        st_.wait_stream(stream)
+    e2e_loop(n_e2e)
+    for st_ in (s_in, s_c, s_out):
+        stream.wait_stream(st_)
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms_rank = e0.elapsed_time(e1) / n_e2e
@@ -364,7 +395,7 @@ def main():
     ap.add_argument("--out", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--transform", default="wush", choices=["wush", "hadamard", "identity"],
                     help="activation-side transform: per-block WUSH (default), one shared Hadamard, or none")
-    ap.add_argument("--ref-rows", type=int, default=2048, help="token rows in the CPU-oracle sample")
+    ap.add_argument("--ref-rows", type=int, default=1024, help="token rows in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -127,15 +127,19 @@ def quantize_act(X, T, fmt, x_tensor_scale=None, sf=SF_LINEAR, out=None):
     return codes, scales
 
 
-def quantize_weight(W, Tinv, fmt, sf=SF_TILED):
-    """W bf16 [N,K], Tinv fp32 [K/g,g,g] -> (codes, scale bytes, w_tensor_scale fp32[1] or None)."""
+def quantize_weight(W, Tinv, fmt, sf=SF_TILED, out=None):
+    """W bf16 [N,K], Tinv fp32 [K/g,g,g] -> (codes, scale bytes, w_tensor_scale fp32[1] or None).
+    `out` = (codes, scales, tensor_scale, workspace) reuses caller-owned buffers."""
     f, g = _fmt(fmt)
     _dev(W, Tinv)
     N, K = W.shape
-    codes, scales = _alloc_q(N, K, g, sf, W.device)
-    ts = torch.zeros(4, dtype=torch.float32, device=W.device) if f == NVFP4 else None
     nws = lib().wush_quantize_weight_workspace_bytes(N, K, f, g)
-    ws = torch.empty(nws, dtype=torch.uint8, device=W.device)
+    if out is not None:
+        codes, scales, ts, ws = out
+    else:
+        codes, scales = _alloc_q(N, K, g, sf, W.device)
+        ts = torch.zeros(4, dtype=torch.float32, device=W.device) if f == NVFP4 else None
+        ws = torch.empty(nws, dtype=torch.uint8, device=W.device)
     check(lib().wush_quantize_weight(_ptr(W), N, K, _ptr(Tinv), f, g, _ptr(ts), _ptr(codes), _ptr(scales), sf,
                                      _ptr(ws), nws, _stream()))
     return codes, scales, ts
@@ -184,7 +188,7 @@ def linear_status(workspace, M, K, g):
     return int(workspace[end - 16:end].view(torch.int32)[0].item())
 
 
-def calib_moments(Xc, g, moments=None, count=None):
+def calib_moments(Xc, g, moments=None, count=None, workspace=None):
     """moments[c] += sum_t x_tc^T x_tc ; count += B.  Returns (moments fp32 [K/g,g,g], count int64[1])."""
     _dev(Xc, moments, count)
     B, K = Xc.shape
@@ -193,7 +197,7 @@ def calib_moments(Xc, g, moments=None, count=None):
     if count is None:
         count = torch.zeros(2, dtype=torch.int64, device=Xc.device)
     nws = lib().wush_calib_moments_workspace_bytes(B, K, g)
-    ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=Xc.device)
+    ws = workspace if workspace is not None else torch.empty(max(nws, 16), dtype=torch.uint8, device=Xc.device)
     check(lib().wush_calib_moments(_ptr(Xc), B, K, g, _ptr(moments), _ptr(count), _ptr(ws), ws.numel(), _stream()))
     return moments, count
 
