@@ -58,7 +58,7 @@ template <int G>
 __global__ void __launch_bounds__(SQ_THREADS, 1)
 tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
                  const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
-                 int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status) {
+                 int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status, int clear_status) {
   constexpr int FMT = (G == 32) ? kFmtMX : kFmtNV;
   extern __shared__ uint8_t sq_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(sq_raw) + 1023) & ~uintptr_t(1023));
@@ -73,6 +73,9 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sq_smem_u32(&empty_bar[s])), "r"(SQ_CONSUMERS));
     }
     *abort_flag = 0;
+    // the status word is only ever set after a bounded wait of about a second has expired, so clearing it
+    // here cannot race with a report; it saves wush_linear a separate memset between kernels
+    if (clear_status && blockIdx.x == 0 && status != nullptr) *status = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -312,7 +315,7 @@ static SqEncodeFn sq_encode_fn() {
 // Returns cudaErrorNotSupported when the streaming kernel cannot take the problem (the caller
 // then uses the register-staged kernel).
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
-                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, cudaStream_t st) {
+                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, cudaStream_t st) {
   SqEncodeFn enc = sq_encode_fn();
   if (!enc) return cudaErrorNotSupported;
   if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
@@ -343,9 +346,9 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   const int grid = (int)(items < sm_count ? items : sm_count);
   const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
   if (g == 32)
-    tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status);
+    tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status, clear_status ? 1 : 0);
   else
-    tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status);
+    tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status, clear_status ? 1 : 0);
   return cudaGetLastError();
 }
 

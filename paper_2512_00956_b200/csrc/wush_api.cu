@@ -79,7 +79,7 @@ int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T, wush_f
   if (!X || !T || !codes || !scales || (fmt == WUSH_NVFP4 && !x_tensor_scale)) return WUSH_ERR_NULL;
   if (!aligned16(X) || !aligned16(T) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
   if (M == 0) return WUSH_OK;
-  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, nullptr, (cudaStream_t)stream);
+  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, nullptr, false, (cudaStream_t)stream);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
@@ -148,10 +148,9 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_
   if (!aligned16(X) || !aligned16(T)) return WUSH_ERR_ALIGN;
   if (M == 0) return WUSH_OK;
   if (!device_is_sm100()) return WUSH_ERR_DEVICE;
-  // one status word for both kernels: cleared here, set by whichever bounded wait expires first
-  cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int32_t), (cudaStream_t)stream);
-  if (e != cudaSuccess) return cuda_fail(e);
-  e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, status, (cudaStream_t)stream);
+  // one status word for both kernels: cleared by the quantiser kernel, set by whichever bounded wait expires
+  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, status, true,
+                                         (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);
   const char* why = nullptr;
   e = wush::run_gemm_fp4(xq, xs, Wcodes, Wscales, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
