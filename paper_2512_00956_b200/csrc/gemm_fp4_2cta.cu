@@ -43,7 +43,8 @@ constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;   // clears the CTA-rank bit of a sh
 __host__ __device__ constexpr int tps(int fmt) { return fmt == kFmtMX ? 2 : 4; }
 __host__ __device__ constexpr int sf_bytes(int fmt) { return 3 * tps(fmt) * 512; }
 __host__ __device__ constexpr int stage_bytes(int fmt) { return A_BYTES + B_BYTES + sf_bytes(fmt); }
-__host__ __device__ constexpr int smem_bytes(int fmt) { return 1024 + STAGES * stage_bytes(fmt) + 256; }
+constexpr int EPI_STAGE_BYTES = 32 * 128;   // per epilogue warp: 32 rows x 128 bytes, 128-byte swizzle
+__host__ __device__ constexpr int smem_bytes(int fmt) { return 1024 + STAGES * stage_bytes(fmt) + EPI_WARPS * EPI_STAGE_BYTES + 256; }
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
@@ -144,7 +145,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                      const __grid_constant__ CUtensorMap mapSFA, const __grid_constant__ CUtensorMap mapSFB,
                      int M, int N, int K, const float* __restrict__ tsx, const float* __restrict__ tsw,
-                     void* __restrict__ Yout, int out_bf16, int32_t* __restrict__ status) {
+                     const __grid_constant__ CUtensorMap mapY, int out_bf16, int32_t* __restrict__ status) {
   constexpr int TPS = tps(FMT);
   constexpr int KSTEPS_PER_TILE = (FMT == kFmtMX) ? 2 : 1;
   extern __shared__ uint8_t raw[];
@@ -152,7 +153,8 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   uint8_t* sA = smem;
   uint8_t* sB = sA + STAGES * A_BYTES;
   uint8_t* sSF = sB + STAGES * B_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sSF + STAGES * sf_bytes(FMT));
+  uint8_t* sEpi = sSF + STAGES * sf_bytes(FMT);     // 1024-byte aligned: all sizes above are multiples of 1 KiB
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sEpi + EPI_WARPS * EPI_STAGE_BYTES);
   uint64_t* full_bar = bars;                      // used in the leader only
   uint64_t* empty_bar = bars + STAGES;            // one copy per CTA, released together by the multicast commit
   uint64_t* tmem_full = bars + 2 * STAGES;        // per CTA
@@ -314,7 +316,6 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++it) {
       const int m0 = (tile / tiles_n) * BM + (int)rank * 128;
       const int n0 = (tile % tiles_n) * BN + half * 128;
-      const int row = m0 + q * 32 + lane;
       if (!__all_sync(0xffffffffu, wait(s32(tmem_full), it & 1, abort_flag))) {
         if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x140000 | (rank << 15) | (it & 0x7fff)); *abort_flag = 1; }
         ok = false;
@@ -332,38 +333,63 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) arrive_leader(s32(tmem_empty));
+      // Store through shared memory and TMA: the warp writes its 32 rows x 128 bytes (swizzled, so the 16-byte
+      // row pieces of the 32 lanes spread over all banks) and one lane hands the box to the TMA unit, which
+      // writes whole 128-byte lines and clips rows >= M and columns >= N by itself.
+      uint8_t* stage = sEpi + (warp - 2) * EPI_STAGE_BYTES;
+      const uint32_t stage_u32 = s32(stage);
+      const bool rows_ok = (m0 + q * 32) < M;              // warp-uniform
+      auto push_box = [&](int col) {                      // buffer filled: hand it to the TMA unit
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                       ::"l"(&mapY), "r"(col), "r"(m0 + q * 32), "r"(stage_u32) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      };
+      auto buffer_free = [&]() {                          // the previous box has been read out of the buffer
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
+      };
+      uint8_t* my_row = stage + lane * 128;
+      if (out_bf16) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int col = n0 + c * 32;
-        if (row < M && col < N) {
-          if (out_bf16) {
-            __nv_bfloat16* y = reinterpret_cast<__nv_bfloat16*>(Yout) + (int64_t)row * N + col;
+        for (int sub = 0; sub < 2; ++sub) {                 // 64 columns (128 bytes of bf16) per box
+          const int col = n0 + sub * 64;
+          if (rows_ok && col < N) {
+            buffer_free();
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              if (col + 8 * v < N) {
-                uint32_t p[4];
+            for (int j = 0; j < 8; ++j) {                   // chunk j = columns 8j..8j+7 = r[2*sub + j/4][8*(j%4)..]
+              uint32_t p[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[c][8 * v + 2 * e]) * alpha,
-                                                           __uint_as_float(r[c][8 * v + 2 * e + 1]) * alpha);
-                  p[e] = *reinterpret_cast<uint32_t*>(&h);
-                }
-                *reinterpret_cast<uint4*>(y + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * sub + (j >> 2)][8 * (j & 3) + 2 * e]) * alpha,
+                                                         __uint_as_float(r[2 * sub + (j >> 2)][8 * (j & 3) + 2 * e + 1]) * alpha);
+                p[e] = *reinterpret_cast<uint32_t*>(&h);
               }
+              *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
             }
-          } else {
-            float* y = reinterpret_cast<float*>(Yout) + (int64_t)row * N + col;
+            push_box(col);
+          }
+        }
+      } else {
 #pragma unroll
-            for (int v = 0; v < 8; ++v) {
-              if (col + 4 * v < N)
-                *reinterpret_cast<float4*>(y + 4 * v) =
-                    make_float4(__uint_as_float(r[c][4 * v]) * alpha, __uint_as_float(r[c][4 * v + 1]) * alpha,
-                                __uint_as_float(r[c][4 * v + 2]) * alpha, __uint_as_float(r[c][4 * v + 3]) * alpha);
-            }
+        for (int sub = 0; sub < 4; ++sub) {                 // 32 columns (128 bytes of fp32) per box
+          const int col = n0 + sub * 32;
+          if (rows_ok && col < N) {
+            buffer_free();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) =
+                  make_uint4(__float_as_uint(__uint_as_float(r[sub][4 * j]) * alpha), __float_as_uint(__uint_as_float(r[sub][4 * j + 1]) * alpha),
+                             __float_as_uint(__uint_as_float(r[sub][4 * j + 2]) * alpha), __float_as_uint(__uint_as_float(r[sub][4 * j + 3]) * alpha));
+            push_box(col);
           }
         }
       }
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // every box written before exit
   }
 
   // ---- common exit: nobody leaves while the peer may still touch this CTA's memory or barriers
@@ -413,9 +439,20 @@ static bool map_scales(CUtensorMap* map, const void* base, int64_t total_tiles, 
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// output [M][N] bf16 or fp32; box = 128 bytes x 32 rows, 128-byte swizzle
+static bool map_output(CUtensorMap* map, void* Y, int64_t M, int64_t N, int out_bf16) {
+  const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)N * (out_bf16 ? 2 : 4)};
+  const cuuint32_t box[2] = {(cuuint32_t)(out_bf16 ? 64 : 32), 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc_fn()(map, out_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, Y, dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int FMT>
 static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& sa, const CUtensorMap& sb,
-                               int M, int N, int K, const float* tsx, const float* tsw, void* Y, int out_bf16,
+                               int M, int N, int K, const float* tsx, const float* tsw, const CUtensorMap& y, int out_bf16,
                                int32_t* status, bool pdl, cudaStream_t st) {
   static int clusters = 0;
   cudaError_t e;
@@ -441,7 +478,7 @@ static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const
   const int tiles = ((M + g2::BM - 1) / g2::BM) * ((N + g2::BN - 1) / g2::BN);
   const int nc = tiles < clusters ? tiles : clusters;
   if (!pdl) {
-    g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, Y,
+    g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, y,
                                                                                      out_bf16, status);
     return cudaGetLastError();
   }
@@ -456,7 +493,7 @@ static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, g2::gemm_fp4_2cta_kernel<FMT>, a, b, sa, sb, M, N, K, tsx, tsw, Y, out_bf16, status);
+  return cudaLaunchKernelEx(&cfg, g2::gemm_fp4_2cta_kernel<FMT>, a, b, sa, sb, M, N, K, tsx, tsw, y, out_bf16, status);
 }
 
 // cudaErrorNotSupported: the caller should use the single-CTA kernel.
@@ -465,13 +502,13 @@ cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_
                               int out_bf16, int32_t* status, bool pdl, cudaStream_t st) {
   if (!enc_fn()) return cudaErrorNotSupported;
   const int64_t ktiles = ((K / (fmt == kFmtMX ? 32 : 16)) + 3) / 4;
-  CUtensorMap a, b, sa, sb;
-  if (!map_bytes(&a, Xq, M, K / 2, 128) || !map_bytes(&b, Wq, N, K / 2, 128) ||
+  CUtensorMap a, b, sa, sb, y;
+  if (!map_output(&y, Y, M, N, out_bf16) || !map_bytes(&a, Xq, M, K / 2, 128) || !map_bytes(&b, Wq, N, K / 2, 128) ||
       !map_scales(&sa, Xs, ((M + 127) / 128) * ktiles, g2::tps(fmt)) ||
       !map_scales(&sb, Ws, ((N + 127) / 128) * ktiles, g2::tps(fmt)))
     return cudaErrorNotSupported;
-  if (fmt == kFmtMX) return launch_2cta<kFmtMX>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, pdl, st);
-  return launch_2cta<kFmtNV>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, pdl, st);
+  if (fmt == kFmtMX) return launch_2cta<kFmtMX>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, y, out_bf16, status, pdl, st);
+  return launch_2cta<kFmtNV>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, y, out_bf16, status, pdl, st);
 }
 
 }  // namespace wush
