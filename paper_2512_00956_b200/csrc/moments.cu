@@ -36,7 +36,7 @@ moments_partial_kernel(const __nv_bfloat16* __restrict__ X, int64_t B, int64_t K
     for (int b = 0; b < 4; ++b) acc[a][b][0] = acc[a][b][1] = acc[a][b][2] = acc[a][b][3] = 0.f;
 
   const __nv_bfloat16* col = X + sb * 32 + 8 * tig;
-  constexpr int UNROLL = 4;
+  constexpr int UNROLL = 8;
   for (int64_t t0 = t_begin; t0 < t_end; t0 += 16 * UNROLL) {
     uint4 lo[UNROLL], hi[UNROLL];
 #pragma unroll
