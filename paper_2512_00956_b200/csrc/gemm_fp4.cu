@@ -197,6 +197,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see the two-CTA kernel
 
   if (warp == 0) {
     // ------------------------------------------------------------------ operand producer

@@ -190,6 +190,9 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   cluster_sync();                                  // both CTAs' barriers exist before anything remote touches them
+  // a programmatic dependent (the next layer's quantiser) may be scheduled as SMs free up; it waits for this
+  // whole grid before it touches memory
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 

@@ -73,12 +73,15 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sq_smem_u32(&empty_bar[s])), "r"(SQ_CONSUMERS));
     }
     *abort_flag = 0;
-    // the status word is only ever set after a bounded wait of about a second has expired, so clearing it
-    // here cannot race with a report; it saves wush_linear a separate memset between kernels
-    if (clear_status && blockIdx.x == 0 && status != nullptr) *status = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // Launched as a programmatic dependent (wush_linear does), everything above ran while the previous kernel
+  // of the stream was still draining; nothing it wrote or still reads may be touched before this point.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // the status word is only ever set after a bounded wait of about a second has expired, so clearing it
+  // here cannot race with a report; it saves wush_linear a separate memset between kernels
+  if (clear_status && blockIdx.x == 0 && threadIdx.x == 0 && status != nullptr) *status = 0;
   // let a programmatic dependent (the GEMM of wush_linear) be scheduled as SMs free up; it still waits
   // for this whole grid before reading the codes
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -315,7 +318,8 @@ static SqEncodeFn sq_encode_fn() {
 // Returns cudaErrorNotSupported when the streaming kernel cannot take the problem (the caller
 // then uses the register-staged kernel).
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
-                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, cudaStream_t st) {
+                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl,
+                                    cudaStream_t st) {
   SqEncodeFn enc = sq_encode_fn();
   if (!enc) return cudaErrorNotSupported;
   if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
@@ -345,11 +349,29 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   if (items > 0x7fffffff || M > 0x7fffff00) return cudaErrorNotSupported;
   const int grid = (int)(items < sm_count ? items : sm_count);
   const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
+  const int cs = clear_status ? 1 : 0;
+  const int n_items = (int)items;
+  if (!pdl) {
+    if (g == 32)
+      tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
+    else
+      tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
+    return cudaGetLastError();
+  }
+  // programmatic dependent launch: set-up overlaps the tail of the previous kernel of the stream
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(SQ_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SQ_SMEM;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (g == 32)
-    tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status, clear_status ? 1 : 0);
-  else
-    tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, (int)items, status, clear_status ? 1 : 0);
-  return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
+  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
 }
 
 }  // namespace wush

@@ -79,7 +79,7 @@ int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T, wush_f
   if (!X || !T || !codes || !scales || (fmt == WUSH_NVFP4 && !x_tensor_scale)) return WUSH_ERR_NULL;
   if (!aligned16(X) || !aligned16(T) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
   if (M == 0) return WUSH_OK;
-  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, nullptr, false, (cudaStream_t)stream);
+  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, nullptr, false, false, (cudaStream_t)stream);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
@@ -149,7 +149,7 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_
   if (M == 0) return WUSH_OK;
   if (!device_is_sm100()) return WUSH_ERR_DEVICE;
   // one status word for both kernels: cleared by the quantiser kernel, set by whichever bounded wait expires
-  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, status, true,
+  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, status, true, true,
                                          (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);
   const char* why = nullptr;

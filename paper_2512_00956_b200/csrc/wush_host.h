@@ -9,11 +9,11 @@ namespace wush {
 // clear_status: the kernel zeroes *status itself (wush_linear); otherwise the word is left alone
 cudaError_t run_quantize_act(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                              uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
-                             cudaStream_t st);
+                             bool pdl, cudaStream_t st);
 // streaming (TMA-fed, persistent) variant; cudaErrorNotSupported = problem not covered, use the other kernel
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                     uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
-                                    cudaStream_t st);
+                                    bool pdl, cudaStream_t st);
 cudaError_t run_transform_f32(const void* X, int64_t M, int64_t K, const void* T, int g, bool t_is_f32,
                               float* V, cudaStream_t st);
 cudaError_t run_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv, int g,
