@@ -354,7 +354,11 @@ def run_ours(args):
     roof = {"bound": "tensor", "kernel": "gemm_fp4_2cta_kernel" if M > 128 else "gemm_fp4_kernel", "achieved": gemm_tf, "peak": fp4_peak, "unit": "TFLOP/s",
             "frac": gemm_tf / fp4_peak, "traffic": traffic.get(f"gemm_fp4_2cta_kernel/config{cfg.index}"), "ms": g_ms,
             "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TF/s x 4 (nominal FP4:bf16)",
-            "frac_of_spec_9pf": gemm_tf / 9000.0}
+            "frac_of_spec_9pf": gemm_tf / 9000.0,
+            # the timed graph replays the kernel back to back for milliseconds, i.e. under the power cap: the
+            # sustained bf16 figure x 4 is the like-for-like ceiling; "frac" keeps the stricter burst figure
+            "peak_sustained": peaks["bf16_tflops_sustained"] * 4.0,
+            "frac_of_sustained": gemm_tf / (peaks["bf16_tflops_sustained"] * 4.0)}
     roof_q = {"bound": "hbm", "kernel": "tq_stream_kernel", "achieved": q_gbs, "peak": peaks["hbm_gbs"],
               "unit": "GB/s", "frac": q_gbs / peaks["hbm_gbs"], "traffic": traffic.get(f"tq_stream_kernel/config{cfg.index}"), "ms": q_ms,
               "algorithmic_bytes": q_bytes, "peak_source": peaks["source"], "frac_of_spec_8tbs": q_gbs / 8000.0}
