@@ -14,7 +14,9 @@ Theorem 4.1), the pre-quantisation invariance W x = (W T^-1)(T x), and the
 dequantised product (exact rational arithmetic on tiny shapes).
 
 Parity unpinned (conventions of this build; the paper is silent): the damping
-ratio lambda = 0.01, the floor rule of the MXFP4 shared exponent, the static
-(calibration-time) NVFP4 activation tensor scale, and the fp32 operation order
-of the NVFP4 block scale.
+ratio lambda = 0.01, the choice between the floor rule (default) and the ceil
+rule ("mxfp4_ceil") of the MXFP4 shared exponent, the choice between the static
+(calibration-time, default) and the per-batch NVFP4 activation tensor scale,
+and the fp32 operation order of the NVFP4 block scale.  (Each rule itself is
+pinned: only which one the paper's authors used is not.)
 """

@@ -75,14 +75,23 @@ class PreparedLayer:
         self.w_codes, self.w_scales = Q.quantize(self.wbar32, fmt, self.ts_w)
         self.w_deq = Q.dequantize(self.w_codes, self.w_scales, fmt, self.ts_w)
 
-    def quantize_act(self, X_bits):
-        Xv = F.bf16_bits_to_f64(X_bits)
-        return quantize_transformed(Xv, self.T_hat, self.fmt, self.ts_x)
+    def dynamic_ts_x(self, X_bits):
+        """NVFP4 tensor scale of THIS batch of activations (instead of the static calibration one):
+        AbsMax over all transformed tokens / (6 * 448)."""
+        v32 = transform_blocks(F.bf16_bits_to_f64(X_bits), self.T_hat).astype(F32)
+        return Q.nvfp4_tensor_scale(v32)
 
-    def forward(self, X_bits, rows=None):
-        """Eq. 7.  ``rows`` optionally restricts the output to a subset of tokens."""
+    def quantize_act(self, X_bits, ts_x=None):
+        """(v32, codes, scales) of q(T x); ``ts_x`` overrides the static NVFP4 tensor scale."""
+        Xv = F.bf16_bits_to_f64(X_bits)
+        return quantize_transformed(Xv, self.T_hat, self.fmt, self.ts_x if ts_x is None else ts_x)
+
+    def forward(self, X_bits, rows=None, dynamic=False):
+        """Eq. 7.  ``rows`` optionally restricts the output to a subset of tokens; ``dynamic``
+        takes the NVFP4 activation tensor scale from the whole batch X_bits."""
+        ts_x = self.dynamic_ts_x(X_bits) if dynamic else self.ts_x
         if rows is not None:
             X_bits = np.asarray(X_bits)[rows]
-        _, codes, scales = self.quantize_act(X_bits)
-        xd = Q.dequantize(codes, scales, self.fmt, self.ts_x)
+        _, codes, scales = self.quantize_act(X_bits, ts_x)
+        xd = Q.dequantize(codes, scales, self.fmt, ts_x)
         return dequantized_product(xd, self.w_deq)

@@ -26,25 +26,36 @@ def _blocks(v, g):
 
 
 # ----------------------------------------------------------------------------- MXFP4
-def mx_shared_exponent(amax):
-    """E8M0 exponent e of a block with AbsMax ``amax``: floor(log2 amax) - 2.
+def mx_shared_exponent(amax, rule="floor"):
+    """E8M0 exponent e of a block with AbsMax ``amax``.
 
-    2 is the exponent of the largest power of two E2M1 represents (4 = 2^2), so
-    amax / 2^e lies in [4, 8); values in (6, 8) saturate to 6.  The exponent is
-    clamped to [-127, 127]; an all-zero block gets -127.
+    rule "floor" (the default of this build): e = floor(log2 amax) - 2.  2 is the
+    exponent of the largest power of two E2M1 represents (4 = 2^2), so amax / 2^e
+    lies in [4, 8); values in (6, 8) saturate to 6.
+    rule "ceil": e = ceil(log2(amax / 6)), the smallest exponent for which no element
+    of the block saturates (amax / 2^e in (3, 6]).  With amax = m * 2^ex, m in
+    [0.5, 1), amax / 6 = (m / 0.75) * 2^(ex - 3) and m / 0.75 lies in [2/3, 4/3): the
+    ceiling is ex - 3 when m <= 0.75 and ex - 2 otherwise - no logarithm is evaluated.
+    Either way the exponent is clamped to [-127, 127]; an all-zero block gets -127.
     """
     amax = np.asarray(amax, dtype=np.float64)
-    _, ex = np.frexp(amax)                   # amax = m * 2^ex, m in [0.5,1): floor(log2) = ex-1
-    e = np.clip(ex - 1 - 2, -127, 127)
+    m, ex = np.frexp(amax)                   # amax = m * 2^ex, m in [0.5,1): floor(log2) = ex-1
+    if rule == "floor":
+        e = ex - 1 - 2
+    elif rule == "ceil":
+        e = ex - 3 + (m > 0.75)
+    else:
+        raise ValueError(rule)
+    e = np.clip(e, -127, 127)
     return np.where(amax == 0, -127, e).astype(np.int64)
 
 
-def quantize_mxfp4(v32):
+def quantize_mxfp4(v32, rule="floor"):
     """fp32 [R, K] -> (codes uint8 [R, K] unpacked, scale bytes uint8 [R, K/32])."""
     v32 = np.asarray(v32, dtype=F32)
     vb = _blocks(v32, 32).astype(np.float64)
     amax = np.max(np.abs(vb), axis=2)
-    e = mx_shared_exponent(amax)
+    e = mx_shared_exponent(amax, rule)
     u = np.ldexp(vb, (-e)[:, :, None])       # exact power-of-two scaling
     codes = F.e2m1_encode(u).reshape(v32.shape)
     return codes, (e + 127).astype(np.uint8)
@@ -57,9 +68,10 @@ def dequantize_mxfp4(codes, scale_bytes):
 
 # ----------------------------------------------------------------------------- NVFP4
 def nvfp4_tensor_scale(v32):
-    """fp32 tensor scale: AbsMax / (6 * 448), one fp32 division."""
+    """fp32 tensor scale: AbsMax / (6 * 448), one fp32 division; 1 for an all-zero tensor
+    (every positive value then gives the same all-zero codes)."""
     amax = F32(np.max(np.abs(np.asarray(v32, dtype=F32)))) if np.size(v32) else F32(0)
-    return F32(amax / F32(2688.0))
+    return F32(1.0) if amax == 0 else F32(amax / F32(2688.0))
 
 
 def quantize_nvfp4(v32, ts):
@@ -93,19 +105,22 @@ def dequantize_nvfp4(codes, scale_bytes, ts):
 
 
 # ----------------------------------------------------------------------------- dispatch
-GROUP = {"mxfp4": 32, "nvfp4": 16}
+# "mxfp4_ceil" is MXFP4 with the non-saturating scale rule; it dequantises like "mxfp4"
+GROUP = {"mxfp4": 32, "nvfp4": 16, "mxfp4_ceil": 32}
 
 
 def quantize(v32, fmt, ts=None):
     if fmt == "mxfp4":
         return quantize_mxfp4(v32)
+    if fmt == "mxfp4_ceil":
+        return quantize_mxfp4(v32, rule="ceil")
     if fmt == "nvfp4":
         return quantize_nvfp4(v32, ts)
     raise ValueError(fmt)
 
 
 def dequantize(codes, scale_bytes, fmt, ts=None):
-    if fmt == "mxfp4":
+    if fmt in ("mxfp4", "mxfp4_ceil"):
         return dequantize_mxfp4(codes, scale_bytes)
     if fmt == "nvfp4":
         return dequantize_nvfp4(codes, scale_bytes, ts)

@@ -156,6 +156,36 @@ def test_mxfp4_scale_rule_properties():
     assert np.all(err[np.abs(u) <= 2] <= 0.25 + 1e-12)
 
 
+def test_mxfp4_ceil_rule_is_the_smallest_non_saturating_exponent():
+    """Exact rationals: e is the least integer with AbsMax <= 6 * 2^e (nothing clamps, nothing is wasted),
+    it is the floor-rule exponent or one more, and the two rules agree exactly when AbsMax / 2^e_floor <= 6."""
+    rng = np.random.default_rng(14)
+    a = np.abs(rng.standard_normal(4000) * np.exp(rng.uniform(-30, 30, 4000))).astype(np.float32)
+    edge = np.float32([6.0, 3.0, 1.5, 0.75, 4.0, 8.0, 12.0, 96.0])           # on and around the decision boundaries
+    edge = np.concatenate([edge, np.nextafter(edge, np.float32(0)), np.nextafter(edge, np.float32(np.inf))])
+    a = np.concatenate([a, edge]).astype(np.float32)
+    e_c = Q.mx_shared_exponent(a, "ceil")
+    e_f = Q.mx_shared_exponent(a, "floor")
+    for x, ec, ef in zip(a, e_c, e_f):
+        fx = Fraction(float(x))
+        assert fx <= 6 * Fraction(2) ** int(ec) and fx > 6 * Fraction(2) ** (int(ec) - 1)
+        assert ec - ef == (1 if fx > 6 * Fraction(2) ** int(ef) else 0)
+    # whole quantiser: no element saturates, so every element is within half a grid step of its value
+    v = (rng.standard_normal((32, 128)) * np.exp(rng.uniform(-10, 10, (32, 1)))).astype(np.float32)
+    codes, sc = Q.quantize(v, "mxfp4_ceil")
+    u = v.reshape(32, 4, 32) / F.e8m0_decode(sc)[:, :, None]
+    assert np.abs(u).max() <= 6.0 and np.all(np.abs(u).max(axis=2) > 3.0)
+    deq_u = Q.dequantize(codes, sc, "mxfp4_ceil").reshape(32, 4, 32) / F.e8m0_decode(sc)[:, :, None]
+    assert np.all(np.abs(deq_u - u) <= 1.0 + 1e-12) and np.all(np.abs(deq_u - u)[np.abs(u) <= 2] <= 0.25 + 1e-12)
+    # worked blocks: AbsMax 6 -> e = 0 under both rules; AbsMax 7 -> floor keeps e = 0 and clamps, ceil takes e = 1
+    blk = np.zeros((1, 32), dtype=np.float32); blk[0, 0] = 7.0; blk[0, 1] = 1.0
+    cf, sf = Q.quantize(blk, "mxfp4"); cc, sc2 = Q.quantize(blk, "mxfp4_ceil")
+    assert sf[0, 0] == 127 and Q.dequantize(cf, sf, "mxfp4")[0, 0] == 6.0
+    assert sc2[0, 0] == 128 and Q.dequantize(cc, sc2, "mxfp4_ceil")[0, 0] == 8.0 and Q.dequantize(cc, sc2, "mxfp4_ceil")[0, 1] == 1.0
+    z = np.zeros((1, 32), dtype=np.float32)
+    assert Q.quantize(z, "mxfp4_ceil")[1][0, 0] == 0
+
+
 def test_nvfp4_worked_block_and_tensor_scale():
     blk = np.zeros((1, 16), dtype=np.float32)
     blk[0, :4] = [6, -3, 1, 0.5]
@@ -168,6 +198,7 @@ def test_nvfp4_worked_block_and_tensor_scale():
     z = np.zeros((1, 16), dtype=np.float32); z[0, 3] = -0.0
     codes, sb = Q.quantize_nvfp4(z, ts)
     assert sb[0, 0] == 0 and np.all((codes & 7) == 0) and codes[0, 3] == 8
+    assert Q.nvfp4_tensor_scale(np.zeros((4, 16), dtype=np.float32)) == np.float32(1.0)   # all-zero tensor: any positive scale
 
 
 def test_nvfp4_matches_exact_rational_definition():

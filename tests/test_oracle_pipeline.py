@@ -91,6 +91,37 @@ def test_forward_close_to_unquantised(fmt, level):
     assert np.allclose(L.forward(d["X"], rows=rows), Y[rows], rtol=1e-12, atol=1e-12)
 
 
+def test_switches_ceil_rule_and_dynamic_tensor_scale():
+    """The two optional rules run through the same pipeline.  Ceil rule: no transformed activation or weight
+    saturates.  Per-batch NVFP4 scale: the block that holds the batch's AbsMax uses the top E4M3 scale (448),
+    a batch 100x larger than the calibration data still quantises without clipping (the static scale clips it),
+    and restricting the output rows does not change the scale."""
+    d, L = _small_layer("mxfp4_ceil", M=64, N=96, K=512, B=512)
+    v32, codes, scales = L.quantize_act(d["X"])
+    assert np.abs(v32.reshape(64, 16, 32) / F.e8m0_decode(scales)[:, :, None]).max() <= 6.0
+    assert np.abs(L.wbar32.reshape(96, 16, 32) / F.e8m0_decode(L.w_scales)[:, :, None]).max() <= 6.0
+    Yref = F.bf16_bits_to_f64(d["X"]) @ F.bf16_bits_to_f64(d["W"]).T
+    rel = np.linalg.norm(L.forward(d["X"]) - Yref) / np.linalg.norm(Yref)
+    assert 0.005 < rel < 0.2
+
+    d, L = _small_layer("nvfp4", M=64, N=96, K=512, B=512)
+    ts = L.dynamic_ts_x(d["X"])
+    _, _, sb = L.quantize_act(d["X"], ts)
+    assert sb.max() == 0x7E
+    Y = L.forward(d["X"], dynamic=True)
+    rows = np.array([3, 17, 40])
+    assert np.allclose(L.forward(d["X"], rows=rows, dynamic=True), Y[rows], rtol=1e-12, atol=1e-12)
+    big = F.f64_to_bf16_bits(F.bf16_bits_to_f64(d["X"]) * 128.0)          # exact in bf16: a power of two
+    Yb_ref = 128.0 * Yref_nv(d)
+    e_dyn = np.linalg.norm(L.forward(big, dynamic=True) - Yb_ref) / np.linalg.norm(Yb_ref)
+    e_sta = np.linalg.norm(L.forward(big) - Yb_ref) / np.linalg.norm(Yb_ref)
+    assert e_dyn < 0.2 and e_sta > 2 * e_dyn
+
+
+def Yref_nv(d):
+    return F.bf16_bits_to_f64(d["X"]) @ F.bf16_bits_to_f64(d["W"]).T
+
+
 def _layer_loss(kind, fmt, d, rng):
     g = Q.GROUP[fmt]
     Xv, Wv, Xc = (F.bf16_bits_to_f64(d[k]) for k in ("X", "W", "Xc"))
