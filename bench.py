@@ -94,14 +94,14 @@ def pick_config(args):
     return cfg, fmt, M
 
 
-def oracle_sample_seconds(cfg, fmt, M, rows):
+def oracle_sample_seconds(cfg, fmt, M, rows, dynamic=False):
     """Times the CPU oracle's online path (transform, quantise, dequantised product) on `rows` tokens."""
     from oracle import pipeline as P
     from paper_2512_00956_b200 import synth
     d = synth.layer_inputs(cfg, M=rows)
     L = P.PreparedLayer(d["W"], d["Xc"], fmt)            # offline part, not timed
     t0 = time.perf_counter()
-    L.forward(d["X"])
+    L.forward(d["X"], dynamic=dynamic)
     return time.perf_counter() - t0
 
 
@@ -125,11 +125,12 @@ def run_reference(args):
     rows = min(M, args.ref_rows)
     d = synth.layer_inputs(cfg, M=rows)
     L = P.PreparedLayer(d["W"], d["Xc"], fmt)
+    dyn = bool(args.dynamic_ts and fmt == "nvfp4")
     for _ in range(args.warmup):
-        L.forward(d["X"])
+        L.forward(d["X"], dynamic=dyn)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        L.forward(d["X"])
+        L.forward(d["X"], dynamic=dyn)
     dt = (time.perf_counter() - t0) / args.steps
     tf = 2.0 * rows * cfg.N * cfg.K / dt / 1e12
     sample = f"{rows} of {M} token rows x all N={cfg.N}, K={cfg.K} per step (fp64 numpy)"
@@ -185,12 +186,19 @@ def run_ours(args):
         d_["xq"] = d_["ws"][: M * K // 2].view(M, K // 2)
         d_["xs"] = d_["ws"][(M * K // 2 + 15) // 16 * 16:][: wush.scale_bytes(M, K, g, wush.SF_TILED)]
 
+    dynamic = bool(args.dynamic_ts and fmt == "nvfp4")
+    ts_step = None if dynamic else layer.x_tensor_scale      # None: wush_linear finds the scale of each batch itself
+    ts_buf = torch.zeros(4, dtype=torch.float32, device=dev)
+
     def step(d_):
-        wush.linear(d_["X"], layer.T, d_["wq"], d_["wsc"], fmt, layer.x_tensor_scale, layer.w_tensor_scale,
+        wush.linear(d_["X"], layer.T, d_["wq"], d_["wsc"], fmt, ts_step, layer.w_tensor_scale,
                     out=d_["Y"], workspace=d_["ws"])
 
     def quant_only(d_):
-        wush.quantize_act(d_["X"], layer.T, fmt, layer.x_tensor_scale, wush.SF_TILED, out=(d_["xq"], d_["xs"]))
+        if dynamic:
+            wush.quantize_act_dynamic(d_["X"], layer.T, wush.SF_TILED, out=(d_["xq"], d_["xs"]), x_tensor_scale=ts_buf)
+        else:
+            wush.quantize_act(d_["X"], layer.T, fmt, layer.x_tensor_scale, wush.SF_TILED, out=(d_["xq"], d_["xs"]))
 
     def gemm_only(d_):
         wush.gemm_fp4(d_["xq"], d_["xs"], d_["wq"], d_["wsc"], K, fmt, layer.x_tensor_scale, layer.w_tensor_scale,
@@ -366,7 +374,7 @@ def run_ours(args):
     cpu = None
     if not args.no_cpu_baseline:
         rows = min(M, args.ref_rows)
-        sec = oracle_sample_seconds(cfg, fmt, M, rows)
+        sec = oracle_sample_seconds(cfg, fmt, M, rows, dynamic)
         cpu = {"value": 2.0 * rows * N * K / sec / 1e12, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
                "sample": f"{rows} of {M} token rows x all N, one pass of the online path (fp64 numpy), {sec:.2f} s"}
 
@@ -374,6 +382,7 @@ def run_ours(args):
             "warmup": max(3, args.warmup), "ms_per_step": t_max * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
             "config": {"workload": cfg.name, "M": M, "K": K, "N": N, "format": fmt, "g": g, "y_dtype": args.out, "transform": args.transform,
+                       "x_tensor_scale": ("per batch" if dynamic else "static") if fmt == "nvfp4" else None,
                        "l2": f"cold data: {nsets} rotating buffer sets of {set_bytes / 1e6:.0f} MB (> 2x L2)",
                        "launch": "one CUDA graph of K steps" if used_graph else "eager loop", "tokens_per_rank": M},
             "roofline": roof, "roofline_quant": roof_q,
@@ -381,7 +390,7 @@ def run_ours(args):
                           "speedup_gemm_only": bf16_ms / g_ms, "impl": "torch.matmul (cuBLAS)"},
             "e2e": {"value": e2e_rate / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": int(X.numel() * 2),
                     "d2h_bytes_per_step": int(Y.numel() * Y.element_size()), "ms_per_step": e2e_ms_rank},
-            "gpu_launches": 2 * args.steps, "kernel_ms": {"transform_quant": q_ms, "gemm_fp4": g_ms},
+            "gpu_launches": (3 if dynamic else 2) * args.steps, "kernel_ms": {"transform_quant": q_ms, "gemm_fp4": g_ms},
             "gemm_status": gemm_status, "offline_kernels": offline, "clocks": clocks, "wall_s_timed_region": wall, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     D.shutdown()
@@ -394,7 +403,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload index 1..5 (2 = the headline configuration)")
-    ap.add_argument("--fmt", default=None, choices=[None, "mxfp4", "nvfp4"])
+    ap.add_argument("--fmt", default=None, choices=[None, "mxfp4", "nvfp4", "mxfp4_ceil"])
+    ap.add_argument("--dynamic-ts", action="store_true",
+                    help="NVFP4: activation tensor scale from each batch (one more kernel per step) instead of calibration")
     ap.add_argument("--m", type=int, default=None, help="override the token count (config 5 sweep)")
     ap.add_argument("--out", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--transform", default="wush", choices=["wush", "hadamard", "identity"],

@@ -57,7 +57,12 @@ typedef enum {
   WUSH_ERR_DEVICE = -8     /* the current device is not compute capability 10.x */
 } wush_status_t;
 
-typedef enum { WUSH_MXFP4 = 0, WUSH_NVFP4 = 1 } wush_format_t;
+/* WUSH_MXFP4_CEIL is MXFP4 with the other common shared-exponent rule (the paper names only
+ * "AbsMax" scaling, Sec. 3): byte = 127 + ceil(log2(AbsMax / 6)), the smallest exponent for
+ * which no element of the block saturates, instead of 127 + floor(log2 AbsMax) - 2.  Codes
+ * and scale bytes have the same meaning, so buffers quantised under either rule feed the
+ * same GEMM; every call that takes a format accepts it with g = 32. */
+typedef enum { WUSH_MXFP4 = 0, WUSH_NVFP4 = 1, WUSH_MXFP4_CEIL = 2 } wush_format_t;
 
 /* Scale-byte layouts.
  *  LINEAR: scales[row][K/g], row-major.
@@ -93,6 +98,18 @@ int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T,
                       wush_format_t fmt, int g, const float* x_tensor_scale,
                       uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf, void* stream);
 
+/* The same step for NVFP4 with the tensor scale taken from THIS batch instead of from calibration
+ * (the paper does not say how the NVFP4 tensor scale of online activations is obtained; the
+ * static one above is this library's default, this is the alternative): a first pass finds
+ * AbsMax over all M x K transformed values, the quantising pass uses AbsMax / (6 * 448)
+ * (1 if the batch is all zero).  X is read twice.
+ *   x_tensor_scale  fp32[2] on the device, WRITTEN: [0] = the scale used (pass it to
+ *          wush_gemm_fp4), [1] = the AbsMax found (also the scratch word of the first pass).
+ * g must be 16.  Errors as wush_quantize_act. */
+int wush_quantize_act_dynamic(const void* X, int64_t M, int64_t K, const void* T, int g,
+                              float* x_tensor_scale, uint8_t* codes, uint8_t* scales,
+                              wush_sf_layout_t sf, void* stream);
+
 /* Offline weight preparation (Algorithm 2, RTN case, last line):
  *   W~ = q( W_blk * Tinv_c^T ),  Tinv = T_xvsh = T_wush^-T (Eq. 6) given in fp32.
  *   W      bf16 [N,K];  Tinv fp32 [K/g][g][g] (same index convention as T above).
@@ -124,7 +141,10 @@ int wush_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const
 /* The whole online layer (Eq. 7): wush_quantize_act into `workspace`, then wush_gemm_fp4,
  * both on `stream`.  Wcodes/Wscales come from wush_quantize_weight with WUSH_SF_TILED.
  * workspace: at least wush_linear_workspace_bytes(M, K, g) bytes, 16-byte aligned.  The
- * last 16 bytes of that region receive the GEMM's status word (see wush_gemm_fp4). */
+ * last 16 bytes of that region receive the GEMM's status word (see wush_gemm_fp4), the 16
+ * bytes before them the activation tensor scale and AbsMax when x_tensor_scale is NULL.
+ * NVFP4 with x_tensor_scale == NULL selects the per-batch tensor scale of
+ * wush_quantize_act_dynamic (one more kernel, X read twice). */
 int wush_linear(const void* X, int64_t M, int64_t K, const void* T,
                 const uint8_t* Wcodes, const uint8_t* Wscales, int64_t N,
                 const float* x_tensor_scale, const float* w_tensor_scale,

@@ -295,6 +295,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after();
+      // *tsx may have been written by the preceding kernel of the stream (per-batch tensor scale).  This
+      // kernel is launched as an ordinary dependent, so the wait returns at once; it keeps the read correct
+      // should the launch ever become a programmatic one
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       float alpha = 1.0f;
       if (FMT == kFmtNV) alpha = __fmul_rn(*tsx, *tsw);
       for (int c = 0; c < BN / 32; ++c) {

@@ -312,6 +312,9 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     // ------------------------------------------------------------------ epilogue (8 warps per CTA)
     const int q = warp & 3;                        // tensor-memory lane quarter this warp may read
     const int half = (warp - 2) >> 2;              // columns [128 half, 128 half + 128)  (warps 2..9)
+    // the activation tensor scale may have been written by the preceding kernel of the stream (per-batch
+    // scale): as a programmatic dependent this grid may read it only after that kernel has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     float alpha = 1.0f;
     if (FMT == kFmtNV) alpha = __fmul_rn(*tsx, *tsw);
     int it = 0;

@@ -58,7 +58,8 @@ template <int G>
 __global__ void __launch_bounds__(SQ_THREADS, 1)
 tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
                  const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
-                 int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status, int clear_status) {
+                 int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status, int clear_status,
+                 const uint32_t* __restrict__ amax_in, float* __restrict__ ts_out, int mx_ceil) {
   constexpr int FMT = (G == 32) ? kFmtMX : kFmtNV;
   extern __shared__ uint8_t sq_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(sq_raw) + 1023) & ~uintptr_t(1023));
@@ -136,7 +137,14 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
     float ts = 1.0f;
-    if (FMT == kFmtNV) ts = *ts_ptr;
+    if (FMT == kFmtNV) {
+      if (amax_in != nullptr) {                 // per-batch tensor scale from the AbsMax pass that ran before
+        ts = nv_tensor_scale(__uint_as_float(*amax_in));
+        if (blockIdx.x == 0 && threadIdx.x == 0 && ts_out != nullptr) *ts_out = ts;
+      } else {
+        ts = *ts_ptr;
+      }
+    }
 
     uint4 tf[2][4];                           // B fragments of the two transforms, kept across items
     int cur_panel = -1;
@@ -221,7 +229,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         }
         float mA, mB;
         if (FMT == kFmtMX) {
-          mx_scale(aA, sA[q], mA); mx_scale(aB, sB[q], mB);
+          mx_scale(aA, sA[q], mA, mx_ceil); mx_scale(aB, sB[q], mB, mx_ceil);
         } else {
           // four distinct scales per quad (row A/B x block 0/1): lane tig computes the one of
           // (row tig>>1, its own block) and fetches the other row's from lane tig^2
@@ -319,7 +327,7 @@ static SqEncodeFn sq_encode_fn() {
 // then uses the register-staged kernel).
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                     uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl,
-                                    cudaStream_t st) {
+                                    cudaStream_t st, const QuantOpts& opt) {
   SqEncodeFn enc = sq_encode_fn();
   if (!enc) return cudaErrorNotSupported;
   if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
@@ -351,11 +359,14 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
   const int cs = clear_status ? 1 : 0;
   const int n_items = (int)items;
+  const uint32_t* amax_in = opt.amax_in;
+  float* ts_out = opt.ts_out;
+  const int mx_ceil = opt.mx_ceil ? 1 : 0;
   if (!pdl) {
     if (g == 32)
-      tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
+      tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
     else
-      tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
+      tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
     return cudaGetLastError();
   }
   // programmatic dependent launch: set-up overlaps the tail of the previous kernel of the stream
@@ -370,8 +381,8 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (g == 32)
-    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
-  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs);
+    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
 }
 
 }  // namespace wush

@@ -17,7 +17,7 @@ int cuda_fail(cudaError_t e, const char* why = nullptr) {
 }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int check_fmt(int fmt, int g) {
-  if (fmt == WUSH_MXFP4) return g == 32 ? WUSH_OK : WUSH_ERR_FORMAT;
+  if (fmt == WUSH_MXFP4 || fmt == WUSH_MXFP4_CEIL) return g == 32 ? WUSH_OK : WUSH_ERR_FORMAT;
   if (fmt == WUSH_NVFP4) return g == 16 ? WUSH_OK : WUSH_ERR_FORMAT;
   return WUSH_ERR_FORMAT;
 }
@@ -28,6 +28,13 @@ inline int check_shape(int64_t rows, int64_t K, int g) {
   return WUSH_OK;
 }
 inline size_t round16(size_t x) { return (x + 15) & ~size_t(15); }
+// the GEMM knows two formats; the scale rule only matters to the quantisers
+inline int gemm_fmt(int fmt) { return fmt == WUSH_NVFP4 ? wush::kFmtNV : wush::kFmtMX; }
+inline wush::QuantOpts opts_of(int fmt) {
+  wush::QuantOpts o;
+  o.mx_ceil = (fmt == WUSH_MXFP4_CEIL);
+  return o;
+}
 
 bool device_is_sm100() {
   static int cached = -1;
@@ -79,7 +86,28 @@ int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T, wush_f
   if (!X || !T || !codes || !scales || (fmt == WUSH_NVFP4 && !x_tensor_scale)) return WUSH_ERR_NULL;
   if (!aligned16(X) || !aligned16(T) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
   if (M == 0) return WUSH_OK;
-  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, nullptr, false, false, (cudaStream_t)stream);
+  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, codes, scales, (int)sf, nullptr, false, false,
+                                         (cudaStream_t)stream, opts_of(fmt));
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+int wush_quantize_act_dynamic(const void* X, int64_t M, int64_t K, const void* T, int g, float* x_tensor_scale,
+                              uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf, void* stream) {
+  int rc = check_fmt(WUSH_NVFP4, g);
+  if (rc) return rc;
+  if ((rc = check_shape(M, K, g))) return rc;
+  if (sf != WUSH_SF_LINEAR && sf != WUSH_SF_TILED) return WUSH_ERR_FORMAT;
+  if (!X || !T || !codes || !scales || !x_tensor_scale) return WUSH_ERR_NULL;
+  if (!aligned16(X) || !aligned16(T) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(x_tensor_scale) & 7u) != 0) return WUSH_ERR_ALIGN;
+  if (M == 0) return WUSH_OK;
+  uint32_t* amax = reinterpret_cast<uint32_t*>(x_tensor_scale + 1);
+  cudaError_t e = wush::run_act_amax(X, M, K, T, amax, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  wush::QuantOpts o;
+  o.amax_in = amax;
+  o.ts_out = x_tensor_scale;
+  e = wush::run_quantize_act(X, M, K, T, g, nullptr, codes, scales, (int)sf, nullptr, false, false, (cudaStream_t)stream, o);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
@@ -98,7 +126,8 @@ int wush_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv,
     return WUSH_ERR_ALIGN;
   if (N == 0) return WUSH_OK;
   cudaError_t e = wush::run_quantize_weight(W, N, K, Tinv, g, w_tensor_scale, codes, scales, (int)sf,
-                                            reinterpret_cast<uint32_t*>(workspace), (cudaStream_t)stream);
+                                            reinterpret_cast<uint32_t*>(workspace), (cudaStream_t)stream,
+                                            fmt == WUSH_MXFP4_CEIL);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
@@ -116,14 +145,15 @@ int wush_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const
   if (M == 0) return WUSH_OK;
   if (!device_is_sm100()) return WUSH_ERR_DEVICE;
   const char* why = nullptr;
-  cudaError_t e = wush::run_gemm_fp4(Xq, Xs, Wq, Ws, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
+  cudaError_t e = wush::run_gemm_fp4(Xq, Xs, Wq, Ws, M, N, K, gemm_fmt(fmt), x_tensor_scale, w_tensor_scale, Y,
                                      ydt == WUSH_OUT_BF16, status, true, false, (cudaStream_t)stream, &why);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e, why);
 }
 
 size_t wush_linear_workspace_bytes(int64_t M, int64_t K, int g) {
   if (M < 0 || K <= 0 || (g != 16 && g != 32) || K % g != 0) return 0;
-  return round16((size_t)(M * (K / 2))) + round16(wush_scale_bytes(M, K, g, WUSH_SF_TILED)) + 16;
+  // packed codes | TILED scale bytes | fp32 tensor scale + AbsMax (per-batch NVFP4 scale) | status word
+  return round16((size_t)(M * (K / 2))) + round16(wush_scale_bytes(M, K, g, WUSH_SF_TILED)) + 16 + 16;
 }
 
 int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_t* Wcodes,
@@ -137,23 +167,34 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_
   if (!aligned16(workspace)) return WUSH_ERR_ALIGN;
   uint8_t* xq = reinterpret_cast<uint8_t*>(workspace);
   uint8_t* xs = xq + round16((size_t)(M * (K / 2)));
-  int32_t* status = reinterpret_cast<int32_t*>(xs + round16(wush_scale_bytes(M, K, g, WUSH_SF_TILED)));
+  float* ts_dyn = reinterpret_cast<float*>(xs + round16(wush_scale_bytes(M, K, g, WUSH_SF_TILED)));
+  int32_t* status = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ts_dyn) + 16);
+  const bool dynamic = (fmt == WUSH_NVFP4 && x_tensor_scale == nullptr);
   // validate the GEMM's arguments before the quantiser touches anything
   if (N <= 0 || N % 8 != 0) return WUSH_ERR_SHAPE;
   if (ydt != WUSH_OUT_F32 && ydt != WUSH_OUT_BF16) return WUSH_ERR_FORMAT;
   if (!X || !T || !Wcodes || !Wscales || !Y) return WUSH_ERR_NULL;
-  if (fmt == WUSH_NVFP4 && (!x_tensor_scale || !w_tensor_scale)) return WUSH_ERR_NULL;
+  if (fmt == WUSH_NVFP4 && !w_tensor_scale) return WUSH_ERR_NULL;
   if (!aligned16(Wcodes) || !aligned16(Wscales) || !aligned16(Y)) return WUSH_ERR_ALIGN;
   if (!X || !T) return WUSH_ERR_NULL;
   if (!aligned16(X) || !aligned16(T)) return WUSH_ERR_ALIGN;
   if (M == 0) return WUSH_OK;
   if (!device_is_sm100()) return WUSH_ERR_DEVICE;
   // one status word for both kernels: cleared by the quantiser kernel, set by whichever bounded wait expires
-  cudaError_t e = wush::run_quantize_act(X, M, K, T, g, x_tensor_scale, xq, xs, WUSH_SF_TILED, status, true, true,
-                                         (cudaStream_t)stream);
+  wush::QuantOpts o = opts_of(fmt);
+  cudaError_t e;
+  if (dynamic) {                                  // per-batch tensor scale: AbsMax pass first
+    uint32_t* amax = reinterpret_cast<uint32_t*>(ts_dyn + 1);
+    if ((e = wush::run_act_amax(X, M, K, T, amax, (cudaStream_t)stream)) != cudaSuccess) return cuda_fail(e);
+    o.amax_in = amax;
+    o.ts_out = ts_dyn;
+    x_tensor_scale = ts_dyn;                      // what the GEMM multiplies by
+  }
+  e = wush::run_quantize_act(X, M, K, T, g, dynamic ? nullptr : x_tensor_scale, xq, xs, WUSH_SF_TILED, status, true, true,
+                             (cudaStream_t)stream, o);
   if (e != cudaSuccess) return cuda_fail(e);
   const char* why = nullptr;
-  e = wush::run_gemm_fp4(xq, xs, Wcodes, Wscales, M, N, K, (int)fmt, x_tensor_scale, w_tensor_scale, Y,
+  e = wush::run_gemm_fp4(xq, xs, Wcodes, Wscales, M, N, K, gemm_fmt(fmt), x_tensor_scale, w_tensor_scale, Y,
                          ydt == WUSH_OUT_BF16, status, false, true, (cudaStream_t)stream, &why);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e, why);
 }
@@ -197,7 +238,8 @@ int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, i
   if (!V || !codes || !scales || (fmt == WUSH_NVFP4 && !tensor_scale)) return WUSH_ERR_NULL;
   if (!aligned16(V) || !aligned16(codes) || !aligned16(scales)) return WUSH_ERR_ALIGN;
   if (R == 0) return WUSH_OK;
-  cudaError_t e = wush::run_quantize_f32(V, R, K, g, tensor_scale, codes, scales, (int)sf, (cudaStream_t)stream);
+  cudaError_t e = wush::run_quantize_f32(V, R, K, g, tensor_scale, codes, scales, (int)sf, (cudaStream_t)stream,
+                                         fmt == WUSH_MXFP4_CEIL);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 

@@ -64,9 +64,14 @@ __device__ __forceinline__ void mul2_rn(float& a, float& b, float m) {
 
 // ---- MXFP4 scale: e = clamp(floor(log2 amax) - 2, -127, 127); returns the E8M0 byte and
 // the exact fp32 multiplier 2^-e.  amax is finite and non-negative.
-__device__ __forceinline__ void mx_scale(float amax, uint32_t& byte, float& mult) {
-  int e = static_cast<int>((__float_as_uint(amax) >> 23) & 0xFF) - 127 - 2;   // zero/subnormal -> -129
-  e = e < -127 ? -127 : e;                                                   // e <= 125 for finite input
+// ceil_rule != 0 selects e = ceil(log2(amax / 6)) instead, the smallest exponent that saturates
+// nothing: with amax = 1.f * 2^E that is E - 2 when the fraction 1.f <= 1.5 and E - 1 otherwise,
+// i.e. the floor-rule exponent plus (mantissa field > 0x400000).
+__device__ __forceinline__ void mx_scale(float amax, uint32_t& byte, float& mult, int ceil_rule = 0) {
+  const uint32_t bits = __float_as_uint(amax);
+  int e = static_cast<int>((bits >> 23) & 0xFF) - 127 - 2;                    // zero/subnormal -> -129
+  if (ceil_rule) e += ((bits & 0x7FFFFFu) > 0x400000u) ? 1 : 0;
+  e = e < -127 ? -127 : e;                                                   // e <= 126 for finite input
   byte = static_cast<uint32_t>(e + 127);
   mult = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);               // 2^-e, biased 2..254
 }
@@ -74,6 +79,12 @@ __device__ __forceinline__ void mx_scale(float amax, uint32_t& byte, float& mult
 __device__ __forceinline__ float e4m3_to_float(uint32_t byte) {
   __half_raw h = __nv_cvt_fp8_to_halfraw(static_cast<__nv_fp8_storage_t>(byte), __NV_E4M3);
   return __half2float(__half(h));
+}
+
+// NVFP4 tensor scale from the AbsMax of the whole tensor: AbsMax / (6 * 448), one fp32 division;
+// 1 for an all-zero tensor (any positive value then yields the same all-zero codes).
+__device__ __forceinline__ float nv_tensor_scale(float amax) {
+  return amax == 0.0f ? 1.0f : __fdiv_rn(amax, 2688.0f);
 }
 
 // ---- NVFP4 scale.  Single-rounded fp32 steps, in this order and with no contraction:

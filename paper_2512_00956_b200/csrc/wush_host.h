@@ -6,21 +6,30 @@
 
 namespace wush {
 
+// Optional rules of the activation quantiser.  mx_ceil: MXFP4 exponent by the ceil rule.  amax_in / ts_out
+// (NVFP4): take the tensor scale from *amax_in (bit pattern of the AbsMax found by run_act_amax) instead of
+// `ts`, and write the scale used to *ts_out.
+struct QuantOpts {
+  bool mx_ceil = false;
+  const uint32_t* amax_in = nullptr;
+  float* ts_out = nullptr;
+};
 // clear_status: the kernel zeroes *status itself (wush_linear); otherwise the word is left alone
 cudaError_t run_quantize_act(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                              uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
-                             bool pdl, cudaStream_t st);
+                             bool pdl, cudaStream_t st, const QuantOpts& opt = QuantOpts());
+cudaError_t run_act_amax(const void* X, int64_t M, int64_t K, const void* T, uint32_t* amax, cudaStream_t st);
 // streaming (TMA-fed, persistent) variant; cudaErrorNotSupported = problem not covered, use the other kernel
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                     uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
-                                    bool pdl, cudaStream_t st);
+                                    bool pdl, cudaStream_t st, const QuantOpts& opt = QuantOpts());
 cudaError_t run_transform_f32(const void* X, int64_t M, int64_t K, const void* T, int g, bool t_is_f32,
                               float* V, cudaStream_t st);
 cudaError_t run_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv, int g,
                                 float* ts_out, uint8_t* codes, uint8_t* scales, int sf,
-                                uint32_t* amax_ws, cudaStream_t st);
+                                uint32_t* amax_ws, cudaStream_t st, bool mx_ceil = false);
 cudaError_t run_quantize_f32(const float* V, int64_t R, int64_t K, int g, const float* ts,
-                             uint8_t* codes, uint8_t* scales, int sf, cudaStream_t st);
+                             uint8_t* codes, uint8_t* scales, int sf, cudaStream_t st, bool mx_ceil = false);
 
 int moments_splits(int64_t B, int64_t K);
 cudaError_t run_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* moments,

@@ -48,7 +48,7 @@ CONFIGS = {
                    m_sweep=(1, 16, 128, 1024, 4096, 16384)),
 }
 
-GROUP = {"mxfp4": 32, "nvfp4": 16}
+GROUP = {"mxfp4": 32, "nvfp4": 16, "mxfp4_ceil": 32}
 
 
 def to_bf16_bits(x):

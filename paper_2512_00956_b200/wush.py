@@ -15,17 +15,17 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwush.so")
 
-MXFP4, NVFP4 = 0, 1
+MXFP4, NVFP4, MXFP4_CEIL = 0, 1, 2
 SF_LINEAR, SF_TILED = 0, 1
 OUT_F32, OUT_BF16 = 0, 1
-FORMATS = {"mxfp4": (MXFP4, 32), "nvfp4": (NVFP4, 16)}
+FORMATS = {"mxfp4": (MXFP4, 32), "nvfp4": (NVFP4, 16), "mxfp4_ceil": (MXFP4_CEIL, 32)}
 
 EXPORTS = [
     "wush_status_string", "wush_last_cuda_error", "wush_scale_bytes", "wush_quantize_act",
     "wush_quantize_weight", "wush_quantize_weight_workspace_bytes", "wush_gemm_fp4", "wush_linear",
     "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
-    "wush_build_transforms",
+    "wush_build_transforms", "wush_quantize_act_dynamic",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -50,6 +50,7 @@ def lib():
         L.wush_scale_bytes.restype = sz
         L.wush_scale_bytes.argtypes = [i64, i64, i32, i32]
         L.wush_quantize_act.argtypes = [vp, i64, i64, vp, i32, i32, vp, vp, vp, i32, vp]
+        L.wush_quantize_act_dynamic.argtypes = [vp, i64, i64, vp, i32, vp, vp, vp, i32, vp]
         L.wush_quantize_weight.argtypes = [vp, i64, i64, vp, i32, i32, vp, vp, vp, i32, vp, sz, vp]
         L.wush_quantize_weight_workspace_bytes.restype = sz
         L.wush_quantize_weight_workspace_bytes.argtypes = [i64, i64, i32, i32]
@@ -93,7 +94,7 @@ def _stream():
 
 
 def _fmt(fmt):
-    return FORMATS[fmt] if isinstance(fmt, str) else (fmt, 32 if fmt == MXFP4 else 16)
+    return FORMATS[fmt] if isinstance(fmt, str) else (fmt, 16 if fmt == NVFP4 else 32)
 
 
 def _dev(*ts):
@@ -125,6 +126,16 @@ def quantize_act(X, T, fmt, x_tensor_scale=None, sf=SF_LINEAR, out=None):
     check(lib().wush_quantize_act(_ptr(X), M, K, _ptr(T), f, g, _ptr(x_tensor_scale), _ptr(codes), _ptr(scales),
                                   sf, _stream()))
     return codes, scales
+
+
+def quantize_act_dynamic(X, T, sf=SF_LINEAR, out=None, x_tensor_scale=None):
+    """NVFP4 with the tensor scale of this batch.  Returns (codes, scale bytes, fp32[2] = scale used, AbsMax)."""
+    _dev(X, T)
+    M, K = X.shape
+    codes, scales = out if out is not None else _alloc_q(M, K, 16, sf, X.device)
+    ts = x_tensor_scale if x_tensor_scale is not None else torch.zeros(4, dtype=torch.float32, device=X.device)
+    check(lib().wush_quantize_act_dynamic(_ptr(X), M, K, _ptr(T), 16, _ptr(ts), _ptr(codes), _ptr(scales), sf, _stream()))
+    return codes, scales, ts
 
 
 def quantize_weight(W, Tinv, fmt, sf=SF_TILED, out=None):
@@ -166,7 +177,8 @@ def linear_workspace_bytes(M, K, g):
 
 def linear(X, T, Wcodes, Wscales, fmt, x_tensor_scale=None, w_tensor_scale=None, out_dtype=torch.float32,
            out=None, workspace=None):
-    """The whole online layer: Y = q(X T^T) (x) W~ (Eq. 7).  Returns (Y, workspace)."""
+    """The whole online layer: Y = q(X T^T) (x) W~ (Eq. 7).  Returns (Y, workspace).
+    NVFP4 with x_tensor_scale=None takes the activation tensor scale from this batch (see linear_dynamic_scale)."""
     f, g = _fmt(fmt)
     _dev(X, T, Wcodes, Wscales)
     M, K = X.shape
@@ -179,6 +191,13 @@ def linear(X, T, Wcodes, Wscales, fmt, x_tensor_scale=None, w_tensor_scale=None,
     check(lib().wush_linear(_ptr(X), M, K, _ptr(T), _ptr(Wcodes), _ptr(Wscales), N, _ptr(x_tensor_scale),
                             _ptr(w_tensor_scale), f, g, _ptr(Y), ydt, _ptr(workspace), workspace.numel(), _stream()))
     return Y, workspace
+
+
+def linear_dynamic_scale(workspace, M, K, g):
+    """(scale used, AbsMax) that an NVFP4 wush_linear call without x_tensor_scale left in its workspace.  Synchronises."""
+    end = linear_workspace_bytes(M, K, g)
+    v = workspace[end - 32:end - 24].view(torch.float32)
+    return float(v[0].item()), float(v[1].item())
 
 
 def linear_status(workspace, M, K, g):

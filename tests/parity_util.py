@@ -4,7 +4,8 @@ out independently of the library, and the guard-band comparison of codes and sca
 Guard bands (tolerance of the build target): an element is "guarded" when the oracle's
 scaled value u lies within 1e-4 relative of an E2M1 rounding midpoint; a whole block is
 guarded when the quantity that decides its scale byte lies within 1e-4 relative of a
-decision boundary (a power of two for MXFP4; an E4M3 rounding midpoint for NVFP4).
+decision boundary (a power of two for MXFP4, 6 times a power of two under its ceil rule; an E4M3
+rounding midpoint for NVFP4).
 Outside the guards codes and scale bytes must be identical; inside, one step apart at most.
 """
 import numpy as np
@@ -57,10 +58,13 @@ def guards(v32, fmt, ts):
     R, K = v32.shape
     vb = v32.reshape(R, K // g, g)
     amax = np.abs(vb).max(axis=2).astype(np.float64)
-    if fmt == "mxfp4":
+    if fmt in ("mxfp4", "mxfp4_ceil"):
         m, _ = np.frexp(np.where(amax == 0, 1.0, amax))              # m in [0.5, 1)
-        block_guard = (m - 0.5 <= 0.5 * GUARD) | (1.0 - m <= GUARD)
-        e = Q.mx_shared_exponent(amax)
+        if fmt == "mxfp4":
+            block_guard = (m - 0.5 <= 0.5 * GUARD) | (1.0 - m <= GUARD)
+        else:                                                        # the exponent steps where AbsMax = 6 * 2^k
+            block_guard = np.abs(m - 0.75) <= 0.75 * GUARD
+        e = Q.mx_shared_exponent(amax, "floor" if fmt == "mxfp4" else "ceil")
         u = np.ldexp(vb.astype(np.float64), (-e)[:, :, None])
     else:
         f32 = np.float32

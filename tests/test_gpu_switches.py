@@ -1,0 +1,124 @@
+"""GPU parity of the two optional quantiser rules against the oracle, through the C ABI:
+the MXFP4 ceil rule ("mxfp4_ceil") and the per-batch NVFP4 activation tensor scale.
+Same tolerances as the main parity tests."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import formats as F
+from oracle import pipeline as P
+from oracle import quantizers as Q
+from paper_2512_00956_b200 import synth, wush
+from parity_util import compare_quantized, dev, dev_bf16, rel_fro, untile
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer(idx, fmt, M=None, N=None, K=None, B=None):
+    d = synth.layer_inputs(synth.CONFIGS[idx], M=M, N=N, K=K, B=B)
+    return d, P.PreparedLayer(d["W"], d["Xc"], fmt)
+
+
+# ------------------------------------------------------------------ MXFP4, ceil rule
+@pytest.mark.parametrize("sf", [wush.SF_LINEAR, wush.SF_TILED])
+def test_ceil_rule_quantize_f32_bit_exact(sf):
+    rng = np.random.default_rng(21)
+    R, K = 333, 512
+    v = (rng.standard_normal((R, K)) * np.exp(rng.uniform(-20, 20, (R, K // 32, 1)).repeat(32, 2).reshape(R, K))).astype(np.float32)
+    v[0, :32] = 0.0
+    v[1, :32] = 0; v[1, 0] = 48.0                                        # AbsMax = 6 * 2^3 exactly: e = 3
+    v[2, :32] = 0; v[2, 5] = -np.nextafter(np.float32(48.0), np.float32(np.inf))   # one ulp above: e = 4
+    v[3, :32] = np.float32(2.0 ** 5) * (1 - 2.0 ** -24)
+    v[4, :32] = 1e-38
+    v[5, :32] = 3e38
+    v[6, :32] = 0; v[6, :7] = [6, 5, 3.5, 2.5, 1.75, 0.75, 0.25]         # exact ties at scale 1
+    codes, scales = wush.quantize_f32(dev(v), "mxfp4_ceil", None, sf)
+    torch.cuda.synchronize()
+    sc = scales.cpu().numpy()
+    if sf == wush.SF_TILED:
+        sc = untile(sc, R, K // 32)
+    compare_quantized(codes.cpu().numpy(), sc, v, "mxfp4_ceil", None, strict=True)
+    # and it differs from the floor rule where it should
+    _, sc_floor = Q.quantize(v, "mxfp4")
+    assert 0.2 < np.mean(sc != sc_floor) < 0.8
+
+
+@pytest.mark.parametrize("M,K,sf", [(128, 2048, wush.SF_TILED), (77, 192, wush.SF_LINEAR), (300, 1024, wush.SF_LINEAR), (1, 64, wush.SF_TILED)])
+def test_ceil_rule_quantize_act_parity(M, K, sf):
+    d, L = _layer(1, "mxfp4_ceil", M=M, N=64, K=K, B=256)
+    codes, scales = wush.quantize_act(dev_bf16(d["X"]), dev_bf16(L.T_bits), "mxfp4_ceil", None, sf)
+    torch.cuda.synchronize()
+    sc = scales.cpu().numpy()
+    if sf == wush.SF_TILED:
+        sc = untile(sc, M, K // 32)
+    v32, _, _ = L.quantize_act(d["X"])
+    stats = compare_quantized(codes.cpu().numpy(), sc, v32, "mxfp4_ceil")
+    assert stats["flipped_codes"] <= stats["guarded_elems"]
+
+
+def test_ceil_rule_weights_and_whole_layer():
+    d, L = _layer(1, "mxfp4_ceil", M=260, N=520, K=1024, B=256)
+    W, X = dev_bf16(d["W"]), dev_bf16(d["X"])
+    wq, ws, _ = wush.quantize_weight(W, dev(L.T_xvsh32), "mxfp4_ceil", sf=wush.SF_LINEAR)
+    torch.cuda.synchronize()
+    compare_quantized(wq.cpu().numpy(), ws.cpu().numpy(), L.wbar32, "mxfp4_ceil")
+    wq, ws, _ = wush.quantize_weight(W, dev(L.T_xvsh32), "mxfp4_ceil", sf=wush.SF_TILED)
+    Y, wsp = wush.linear(X, dev_bf16(L.T_bits), wq, ws, "mxfp4_ceil")
+    torch.cuda.synchronize()
+    assert wush.linear_status(wsp, 260, 1024, 32) == 0
+    assert rel_fro(Y.cpu().numpy(), L.forward(d["X"])) <= 1e-3
+    # the GEMM does not care which rule produced its operands
+    xq, xs = wush.quantize_act(X, dev_bf16(L.T_bits), "mxfp4_ceil", None, wush.SF_TILED)
+    Y2, st = wush.gemm_fp4(xq, xs, wq, ws, 1024, "mxfp4")
+    torch.cuda.synchronize()
+    assert int(st[0].item()) == 0 and torch.equal(Y, Y2)
+
+
+# ------------------------------------------------------------------ NVFP4, per-batch tensor scale
+@pytest.mark.parametrize("M,K,sf", [(128, 2048, wush.SF_TILED), (77, 320, wush.SF_LINEAR), (531, 1024, wush.SF_TILED), (16, 64, wush.SF_LINEAR)])
+def test_dynamic_scale_quantize_act_parity(M, K, sf):
+    d, L = _layer(2, "nvfp4", M=M, N=64, K=K, B=256)
+    codes, scales, ts = wush.quantize_act_dynamic(dev_bf16(d["X"]), dev_bf16(L.T_bits), sf)
+    torch.cuda.synchronize()
+    ts_o = L.dynamic_ts_x(d["X"])
+    ts_g, amax_g = (float(x) for x in ts.cpu().numpy()[:2])
+    assert abs(ts_g - float(ts_o)) <= 2e-7 * float(ts_o)
+    assert np.float32(ts_g) == np.float32(np.float32(amax_g) / np.float32(2688.0))
+    sc = scales.cpu().numpy()
+    if sf == wush.SF_TILED:
+        sc = untile(sc, M, K // 16)
+    v32, _, _ = L.quantize_act(d["X"], ts_o)
+    compare_quantized(codes.cpu().numpy(), sc, v32, "nvfp4", ts_o)
+    assert sc.max() == 0x7E                                   # the AbsMax block uses the top E4M3 scale
+
+
+@pytest.mark.parametrize("M,N,K", [(77, 136, 320), (300, 520, 1024), (1, 64, 64)])
+def test_dynamic_scale_whole_layer(M, N, K):
+    d, L = _layer(2, "nvfp4", M=M, N=N, K=K, B=256)
+    W, X = dev_bf16(d["W"]), dev_bf16(d["X"])
+    wq, ws, tsw = wush.quantize_weight(W, dev(L.T_xvsh32), "nvfp4", sf=wush.SF_TILED)
+    Y, wsp = wush.linear(X, dev_bf16(L.T_bits), wq, ws, "nvfp4", None, tsw)          # no x_tensor_scale: per batch
+    torch.cuda.synchronize()
+    assert wush.linear_status(wsp, M, K, 16) == 0
+    ts_g, _ = wush.linear_dynamic_scale(wsp, M, K, 16)
+    ts_o = float(L.dynamic_ts_x(d["X"]))
+    assert abs(ts_g - ts_o) <= 2e-7 * ts_o
+    assert rel_fro(Y.cpu().numpy(), L.forward(d["X"], dynamic=True)) <= 1e-3
+    # a batch far outside the calibration range: the static scale clips, the per-batch one does not
+    big = F.f64_to_bf16_bits(F.bf16_bits_to_f64(d["X"]) * 128.0)
+    Yb, wsp = wush.linear(dev_bf16(big), dev_bf16(L.T_bits), wq, ws, "nvfp4", None, tsw, workspace=wsp)
+    torch.cuda.synchronize()
+    assert rel_fro(Yb.cpu().numpy(), L.forward(big, dynamic=True)) <= 1e-3
+    # second call on the same workspace, same input: identical (nothing is left over between calls)
+    Yb2, _ = wush.linear(dev_bf16(big), dev_bf16(L.T_bits), wq, ws, "nvfp4", None, tsw, workspace=wsp)
+    torch.cuda.synchronize()
+    assert torch.equal(Yb, Yb2)
+
+
+def test_dynamic_scale_all_zero_batch():
+    d, L = _layer(2, "nvfp4", M=40, N=64, K=128, B=256)
+    X = torch.zeros(40, 128, dtype=torch.bfloat16, device="cuda")
+    codes, scales, ts = wush.quantize_act_dynamic(X, dev_bf16(L.T_bits), wush.SF_LINEAR)
+    torch.cuda.synchronize()
+    assert float(ts[0].item()) == 1.0 and float(ts[1].item()) == 0.0
+    assert int(codes.max().item()) == 0 and int(scales.max().item()) == 0

@@ -41,7 +41,7 @@ def test_scale_bytes(L):
     assert L.wush_scale_bytes(129, 64, 32, wush.SF_TILED) == 2 * 1 * 512
     assert L.wush_scale_bytes(1, 64, 16, wush.SF_TILED) == 512
     assert L.wush_scale_bytes(1, 64, 8, wush.SF_TILED) == 0
-    assert L.wush_linear_workspace_bytes(128, 2048, 32) == 128 * 1024 + 16 * 512 + 16
+    assert L.wush_linear_workspace_bytes(128, 2048, 32) == 128 * 1024 + 16 * 512 + 16 + 16   # codes, scales, tensor scale slot, status
     assert L.wush_calib_moments_workspace_bytes(512, 2048, 32) % (2048 * 32 * 4) == 0
 
 
