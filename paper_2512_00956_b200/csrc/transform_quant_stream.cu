@@ -54,7 +54,10 @@ __device__ __forceinline__ bool sq_elect() {
   return pred != 0;
 }
 
-template <int G>
+// AMAX = true: the same tile walk and the same products, but instead of quantising, the AbsMax of everything
+// computed is folded into *ts_out (read as the uint32 bit pattern of a non-negative float, atomicMax): the
+// first pass of the per-batch NVFP4 tensor scale.  codes / scales are not touched.
+template <int G, bool AMAX = false>
 __global__ void __launch_bounds__(SQ_THREADS, 1)
 tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
                  const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
@@ -137,7 +140,8 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
     float ts = 1.0f;
-    if (FMT == kFmtNV) {
+    float seen = 0.0f;                         // AMAX: running maximum of this lane
+    if (FMT == kFmtNV && !AMAX) {
       if (amax_in != nullptr) {                 // per-batch tensor scale from the AbsMax pass that ran before
         ts = nv_tensor_scale(__uint_as_float(*amax_in));
         if (blockIdx.x == 0 && threadIdx.x == 0 && ts_out != nullptr) *ts_out = ts;
@@ -221,6 +225,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         float aB = fmaxf(fmaxf(fabsf(vB[0]), fabsf(vB[1])), fabsf(vB[2]));
         aB = fmaxf(fmaxf(aB, fabsf(vB[3])), fabsf(vB[4]));
         aB = fmaxf(fmaxf(aB, fabsf(vB[5])), fmaxf(fabsf(vB[6]), fabsf(vB[7])));
+        if (AMAX) { seen = fmaxf(seen, fmaxf(okA ? aA : 0.0f, okB ? aB : 0.0f)); continue; }
         aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 2));       // lanes tig and tig^2 share a g=16 block
         aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 2));
         if (G == 32) {
@@ -246,6 +251,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         wA[q] = pack_e2m1x8_fast(vA);
         wB[q] = pack_e2m1x8_fast(vB);
       }
+      if (AMAX) continue;
       // ---- codes: lanes 0,1 gather super-block 0, lanes 2,3 super-block 1 (8 contiguous bytes each)
       {
         const bool lo = tig < 2;
@@ -302,6 +308,11 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         }
       }
     }
+    if (AMAX) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) seen = fmaxf(seen, __shfl_xor_sync(0xffffffffu, seen, o));
+      if (lane == 0 && ts_out != nullptr) atomicMax(reinterpret_cast<uint32_t*>(ts_out), __float_as_uint(seen));
+    }
   }
   __syncthreads();
 }
@@ -349,6 +360,7 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
     if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(tq_stream_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(tq_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
     attr_done = true;
   }
   const int num_rb = (int)((M + SQ_ROWS - 1) / SQ_ROWS);
@@ -362,6 +374,12 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   const uint32_t* amax_in = opt.amax_in;
   float* ts_out = opt.ts_out;
   const int mx_ceil = opt.mx_ceil ? 1 : 0;
+  if (opt.amax_out != nullptr) {                 // AbsMax pass only (g = 16)
+    if (g != 16) return cudaErrorNotSupported;
+    tq_stream_kernel<16, true><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, nullptr, nullptr, nullptr, sf, num_rb, n_items,
+                                                                  nullptr, 0, nullptr, reinterpret_cast<float*>(opt.amax_out), 0);
+    return cudaGetLastError();
+  }
   if (!pdl) {
     if (g == 32)
       tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
