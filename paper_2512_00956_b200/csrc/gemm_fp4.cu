@@ -205,7 +205,35 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     // uniform registers); one elected lane issues the copies.
     int issued = 0;
     bool ok = true;
-    for (int kb = 0; kb < num_kb; ++kb) {
+    // Weights do not depend on the preceding kernel of the stream.  Launched as a programmatic dependent of
+    // the quantiser, this CTA may start while that kernel still runs: the first ring-full of weight tiles and
+    // weight scales is requested at once, the activation side only after the quantiser has completed.
+    // (The whole stage's byte count is announced with the first half, so the barrier flips when both landed.)
+    const int pre = min(STAGES, num_kb);
+    auto weights = [&](int kb, int s, uint32_t bar, uint32_t sf_bytes) {
+      uint8_t* sf = sSF + s * stage_sf_bytes(FMT);
+      mbar_expect_tx(bar, a_box_bytes + B_BYTES + sf_bytes * 2);
+      tma_load_2d(smem_u32(sB + s * B_BYTES), &mapB, kb * BKB, n0, bar);
+      bulk_load_1d(smem_u32(sf + TPS * 512), SFB + ((int64_t)(n0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
+    };
+    auto activations = [&](int kb, int s, uint32_t bar, uint32_t sf_bytes) {
+      // the A box covers only round_up(M, 8) rows when M < 128: the rows of the stage below it keep stale
+      // bytes, which only reach accumulator rows that are never stored
+      uint8_t* sf = sSF + s * stage_sf_bytes(FMT);
+      tma_load_2d(smem_u32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
+      bulk_load_1d(smem_u32(sf), SFA + ((int64_t)(m0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
+    };
+    if (elect_one())
+      for (int kb = 0; kb < pre; ++kb)
+        weights(kb, kb, smem_u32(&full_bar[kb]), min(TPS, ktiles_total - kb * TPS) * 512);
+    __syncwarp();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (elect_one())
+      for (int kb = 0; kb < pre; ++kb)
+        activations(kb, kb, smem_u32(&full_bar[kb]), min(TPS, ktiles_total - kb * TPS) * 512);
+    __syncwarp();
+    issued = pre;
+    for (int kb = pre; kb < num_kb; ++kb) {
       const int s = kb % STAGES;
       const uint32_t ph = (kb / STAGES) & 1;
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag))) {
@@ -216,18 +244,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         ok = false;
         break;
       }
-      const int tiles = min(TPS, ktiles_total - kb * TPS);
-      const uint32_t sf_bytes = tiles * 512;
+      const uint32_t sf_bytes = min(TPS, ktiles_total - kb * TPS) * 512;
       const uint32_t bar = smem_u32(&full_bar[s]);
-      uint8_t* sf = sSF + s * stage_sf_bytes(FMT);
       if (elect_one()) {
-        // the A box covers only round_up(M, 8) rows when M < 128: the rows of the stage below it keep stale
-        // bytes, which only reach accumulator rows that are never stored
-        mbar_expect_tx(bar, a_box_bytes + B_BYTES + sf_bytes * 2);
-        tma_load_2d(smem_u32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
-        tma_load_2d(smem_u32(sB + s * B_BYTES), &mapB, kb * BKB, n0, bar);
-        bulk_load_1d(smem_u32(sf), SFA + ((int64_t)(m0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
-        bulk_load_1d(smem_u32(sf + TPS * 512), SFB + ((int64_t)(n0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
+        weights(kb, s, bar, sf_bytes);
+        activations(kb, s, bar, sf_bytes);
       }
       __syncwarp();
       ++issued;
@@ -295,9 +316,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after();
-      // *tsx may have been written by the preceding kernel of the stream (per-batch tensor scale).  This
-      // kernel is launched as an ordinary dependent, so the wait returns at once; it keeps the read correct
-      // should the launch ever become a programmatic one
+      // *tsx may have been written by the preceding kernel of the stream (per-batch tensor scale); as a
+      // programmatic dependent this grid may read it only after that kernel has completed
       asm volatile("griddepcontrol.wait;" ::: "memory");
       float alpha = 1.0f;
       if (FMT == kFmtNV) alpha = __fmul_rn(*tsx, *tsw);
@@ -396,6 +416,16 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
     return cudaErrorInvalidValue;
   }
   dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = after_quantizer ? 1 : 0;          // programmatic dependent of the quantiser inside wush_linear
+  const int mi = (int)M, ni = (int)N, ki = (int)K, a_bytes = a_rows * BKB;
   if (fmt == kFmtMX) {
     static bool attr_done = false;
     if (!attr_done) {
@@ -403,19 +433,17 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
       if (e != cudaSuccess) return e;
       attr_done = true;
     }
-    gemm_fp4_kernel<kFmtMX><<<grid, GEMM_THREADS, gemm_smem_bytes(kFmtMX), st>>>(
-        mapA, mapB, Xs, Ws, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, a_rows * BKB);
-  } else {
-    static bool attr_done = false;
-    if (!attr_done) {
-      e = cudaFuncSetAttribute(gemm_fp4_kernel<kFmtNV>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(kFmtNV));
-      if (e != cudaSuccess) return e;
-      attr_done = true;
-    }
-    gemm_fp4_kernel<kFmtNV><<<grid, GEMM_THREADS, gemm_smem_bytes(kFmtNV), st>>>(
-        mapA, mapB, Xs, Ws, (int)M, (int)N, (int)K, tsx, tsw, Y, out_bf16, status, a_rows * BKB);
+    cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtMX);
+    return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtMX>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes);
   }
-  return cudaGetLastError();
+  static bool attr_done = false;
+  if (!attr_done) {
+    e = cudaFuncSetAttribute(gemm_fp4_kernel<kFmtNV>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(kFmtNV));
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtNV);
+  return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtNV>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes);
 }
 
 }  // namespace wush

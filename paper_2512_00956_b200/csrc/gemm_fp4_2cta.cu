@@ -200,13 +200,42 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     // ------------------------------------------------------------------ producer (one per CTA)
     int g = 0;                                     // running k-block count across tiles
     bool ok = true;
+    // weight side of a stage (the leader also announces the stage's whole byte count), activation side
+    auto weights = [&](int kb, int s, int n0) {
+      const uint32_t bar = s32(&full_bar[s]) & PEER_MASK;            // the leader's barrier
+      if (rank == 0)
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(&full_bar[s])), "r"(2 * stage_bytes(FMT)) : "memory");
+      uint8_t* sf = sSF + s * sf_bytes(FMT);
+      tma_2sm(s32(sB + s * B_BYTES), &mapB, kb * BKB, n0 + (int)rank * 128, bar);
+      tma_2sm(s32(sf + TPS * 512), &mapSFB, 0, (n0 >> 7) * ktiles_total + kb * TPS, bar);
+      tma_2sm(s32(sf + 2 * TPS * 512), &mapSFB, 0, ((n0 >> 7) + 1) * ktiles_total + kb * TPS, bar);
+    };
+    auto activations = [&](int kb, int s, int m0) {
+      const uint32_t bar = s32(&full_bar[s]) & PEER_MASK;
+      uint8_t* sf = sSF + s * sf_bytes(FMT);
+      tma_2sm(s32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
+      tma_2sm(s32(sf), &mapSFA, 0, (m0 >> 7) * ktiles_total + kb * TPS, bar);
+    };
     // Launched as a programmatic dependent of the quantiser (wush_linear), everything above overlapped with
-    // that kernel's tail; its output may be read only after this point.  A no-op for a plain launch.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // that kernel's tail.  The weights do not depend on it: the first ring-full of weight tiles is requested
+    // before the wait, the quantiser's output only after it.  The wait is a no-op for a plain launch.
+    const int pre = (cluster_id < num_tiles) ? min(STAGES, num_kb) : 0;
+    if (pre > 0) {
+      const int m0 = (cluster_id / tiles_n) * BM + (int)rank * 128;
+      const int n0 = (cluster_id % tiles_n) * BN;
+      if (elect())
+        for (int kb = 0; kb < pre; ++kb) weights(kb, kb, n0);
+      __syncwarp();
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (elect())
+        for (int kb = 0; kb < pre; ++kb) activations(kb, kb, m0);
+      __syncwarp();
+    }
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
       const int m0 = (tile / tiles_n) * BM + (int)rank * 128;
       const int n0 = (tile % tiles_n) * BN;
-      for (int kb = 0; kb < num_kb; ++kb, ++g) {
+      for (int kb = (tile == cluster_id ? pre : 0); kb < num_kb; ++kb) {
+        g = ((tile - cluster_id) / num_clusters) * num_kb + kb;
         const int s = g % STAGES;
         const uint32_t ph = (g / STAGES) & 1;
         if (!__all_sync(0xffffffffu, wait(s32(&empty_bar[s]), ph ^ 1, abort_flag))) {
@@ -215,15 +244,8 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
           break;
         }
         if (elect()) {
-          const uint32_t bar = s32(&full_bar[s]) & PEER_MASK;        // the leader's barrier
-          if (rank == 0)
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(&full_bar[s])), "r"(2 * stage_bytes(FMT)) : "memory");
-          uint8_t* sf = sSF + s * sf_bytes(FMT);
-          tma_2sm(s32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
-          tma_2sm(s32(sB + s * B_BYTES), &mapB, kb * BKB, n0 + (int)rank * 128, bar);
-          tma_2sm(s32(sf), &mapSFA, 0, (m0 >> 7) * ktiles_total + kb * TPS, bar);
-          tma_2sm(s32(sf + TPS * 512), &mapSFB, 0, (n0 >> 7) * ktiles_total + kb * TPS, bar);
-          tma_2sm(s32(sf + 2 * TPS * 512), &mapSFB, 0, ((n0 >> 7) + 1) * ktiles_total + kb * TPS, bar);
+          weights(kb, s, n0);
+          activations(kb, s, m0);
         }
         __syncwarp();
       }
