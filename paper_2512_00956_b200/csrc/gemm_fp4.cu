@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const uint8_t* __restrict__ SFA, const uint8_t* __restrict__ SFB, int M, int N, int K,
                 const float* __restrict__ tsx, const float* __restrict__ tsw, void* __restrict__ Yout,
-                int out_bf16, int32_t* __restrict__ status, int a_box_bytes) {
+                int out_bf16, int32_t* __restrict__ status, int a_box_bytes, int clear_status) {
   constexpr int TPS = sf_tiles_per_stage(FMT);           // scale tiles (4 scale columns each) per stage
   constexpr int KSTEPS_PER_TILE = (FMT == kFmtMX) ? 2 : 1;  // K=64 MMAs covered by one scale tile
   extern __shared__ uint8_t smem_raw[];
@@ -183,6 +183,10 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
   const int sf_cols = K / (FMT == kFmtMX ? 32 : 16);
   const int ktiles_total = (sf_cols + 3) >> 2;            // scale tiles along K
 
+  if (threadIdx.x == 64) { prefetch_tensormap(&mapB); prefetch_tensormap(&mapA); }
+  // stand-alone call: the first CTA clears the status word (a report can only follow a wait of about two
+  // seconds, so this cannot erase one); inside wush_linear the quantiser kernel has cleared it
+  if (clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 96 && status != nullptr) *status = 0;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
     mbar_init(smem_u32(tmem_full_bar), 1);
@@ -401,12 +405,9 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
                          void* Y, int out_bf16, int32_t* status, bool clear_status, bool after_quantizer, cudaStream_t st,
                          const char** why) {
   cudaError_t e;
-  if (status && clear_status) {
-    e = cudaMemsetAsync(status, 0, sizeof(int32_t), st);
-    if (e != cudaSuccess) return e;
-  }
+  const int cs = (status && clear_status) ? 1 : 0;
   if (M > 128) {
-    e = run_gemm_fp4_2cta(Xq, Xs, Wq, Ws, M, N, K, fmt, tsx, tsw, Y, out_bf16, status, after_quantizer, st);
+    e = run_gemm_fp4_2cta(Xq, Xs, Wq, Ws, M, N, K, fmt, tsx, tsw, Y, out_bf16, status, cs != 0, after_quantizer, st);
     if (e != cudaErrorNotSupported) return e;
   }
   CUtensorMap mapA, mapB;
@@ -434,7 +435,7 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
       attr_done = true;
     }
     cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtMX);
-    return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtMX>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes);
+    return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtMX>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes, cs);
   }
   static bool attr_done = false;
   if (!attr_done) {
@@ -443,7 +444,7 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
     attr_done = true;
   }
   cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtNV);
-  return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtNV>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes);
+  return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtNV>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes, cs);
 }
 
 }  // namespace wush

@@ -145,7 +145,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                      const __grid_constant__ CUtensorMap mapSFA, const __grid_constant__ CUtensorMap mapSFB,
                      int M, int N, int K, const float* __restrict__ tsx, const float* __restrict__ tsw,
-                     const __grid_constant__ CUtensorMap mapY, int out_bf16, int32_t* __restrict__ status) {
+                     const __grid_constant__ CUtensorMap mapY, int out_bf16, int32_t* __restrict__ status, int clear_status) {
   constexpr int TPS = tps(FMT);
   constexpr int KSTEPS_PER_TILE = (FMT == kFmtMX) ? 2 : 1;
   extern __shared__ uint8_t raw[];
@@ -172,6 +172,13 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   const int sf_cols = K / (FMT == kFmtMX ? 32 : 16);
   const int ktiles_total = (sf_cols + 3) >> 2;
 
+  if (threadIdx.x == 32 * SF_WARP) {             // descriptors on their way while the barriers and TMEM are set up
+    prefetch_tensormap(&mapB); prefetch_tensormap(&mapSFB); prefetch_tensormap(&mapA); prefetch_tensormap(&mapSFA);
+    prefetch_tensormap(&mapY);
+    // stand-alone call: clear the status word here (a report can only follow a wait of about two seconds, so
+    // this cannot erase one); inside wush_linear the quantiser kernel has cleared it
+    if (clear_status && blockIdx.x == 0 && status != nullptr) *status = 0;
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(&full_bar[s])), "r"(1));
@@ -417,7 +424,9 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
         }
       }
     }
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // every box written before exit
+    // every box has been read out of shared memory before the CTA may exit; the writes themselves complete
+    // with the grid
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
   }
 
   // ---- common exit: nobody leaves while the peer may still touch this CTA's memory or barriers
@@ -481,8 +490,9 @@ static bool map_output(CUtensorMap* map, void* Y, int64_t M, int64_t N, int out_
 template <int FMT>
 static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& sa, const CUtensorMap& sb,
                                int M, int N, int K, const float* tsx, const float* tsw, const CUtensorMap& y, int out_bf16,
-                               int32_t* status, bool pdl, cudaStream_t st) {
+                               int32_t* status, bool clear_status, bool pdl, cudaStream_t st) {
   static int clusters = 0;
+  const int cs = clear_status ? 1 : 0;
   cudaError_t e;
   if (clusters == 0) {
     e = cudaFuncSetAttribute(g2::gemm_fp4_2cta_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, g2::smem_bytes(FMT));
@@ -507,7 +517,7 @@ static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const
   const int nc = tiles < clusters ? tiles : clusters;
   if (!pdl) {
     g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, y,
-                                                                                     out_bf16, status);
+                                                                                     out_bf16, status, cs);
     return cudaGetLastError();
   }
   // programmatic dependent launch: this grid may start while the preceding kernel of the stream drains
@@ -521,13 +531,13 @@ static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, g2::gemm_fp4_2cta_kernel<FMT>, a, b, sa, sb, M, N, K, tsx, tsw, y, out_bf16, status);
+  return cudaLaunchKernelEx(&cfg, g2::gemm_fp4_2cta_kernel<FMT>, a, b, sa, sb, M, N, K, tsx, tsw, y, out_bf16, status, cs);
 }
 
 // cudaErrorNotSupported: the caller should use the single-CTA kernel.
 cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws, int64_t M,
                               int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw, void* Y,
-                              int out_bf16, int32_t* status, bool pdl, cudaStream_t st) {
+                              int out_bf16, int32_t* status, bool clear_status, bool pdl, cudaStream_t st) {
   if (!enc_fn()) return cudaErrorNotSupported;
   const int64_t ktiles = ((K / (fmt == kFmtMX ? 32 : 16)) + 3) / 4;
   CUtensorMap a, b, sa, sb, y;
@@ -535,8 +545,8 @@ cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_
       !map_scales(&sa, Xs, ((M + 127) / 128) * ktiles, g2::tps(fmt)) ||
       !map_scales(&sb, Ws, ((N + 127) / 128) * ktiles, g2::tps(fmt)))
     return cudaErrorNotSupported;
-  if (fmt == kFmtMX) return launch_2cta<kFmtMX>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, y, out_bf16, status, pdl, st);
-  return launch_2cta<kFmtNV>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, y, out_bf16, status, pdl, st);
+  if (fmt == kFmtMX) return launch_2cta<kFmtMX>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, y, out_bf16, status, clear_status, pdl, st);
+  return launch_2cta<kFmtNV>(a, b, sa, sb, (int)M, (int)N, (int)K, tsx, tsw, y, out_bf16, status, clear_status, pdl, st);
 }
 
 }  // namespace wush

@@ -71,6 +71,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + SQ_STAGES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 32) prefetch_tensormap(&mapX);
   if (threadIdx.x == 0) {
     for (int s = 0; s < SQ_STAGES; ++s) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sq_smem_u32(&full_bar[s])), "r"(1));
