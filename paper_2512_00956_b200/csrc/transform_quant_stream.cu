@@ -16,6 +16,8 @@
 //    bytes and a row's 32 bytes leave as one full sector per quad.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "wush_device.cuh"
 #include "wush_host.h"
 
@@ -47,6 +49,18 @@ __device__ __forceinline__ bool sq_wait(uint32_t bar, uint32_t parity, volatile 
       if (sq_try_wait(bar, parity)) return true;
     if (*abort_flag != 0 || sq_timer() - t0 > 1000000000ull) return false;
   }
+}
+__device__ __forceinline__ uint4 sq_lds128(uint32_t addr) {          // 128-bit load from a 32-bit shared address
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+// four 8x8 matrices of 16-bit elements, one row address per lane: the result is the A operand of m16n8k16
+__device__ __forceinline__ uint4 sq_ldmatrix_x4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
 }
 __device__ __forceinline__ bool sq_elect() {
   uint32_t pred;
@@ -134,9 +148,15 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     // ------------------------------------------------------------------ consumer warps
     const int gid = lane >> 2, tig = lane & 3;
     const int mt = warp & 7;                  // 16-row slice of the tile
-    // MMA row slot gid reads tile row 16*mt + pi(gid), pi = (0,4,1,5,2,6,3,7): the two rows of a
-    // quarter-warp then differ in bit 2, which the swizzle turns into disjoint bank halves
-    const int prow = 16 * mt + ((gid & 1) << 2) + (gid >> 1);
+    // Two ways to fetch the A operands.  g = 32: ldmatrix, whose four destination registers ARE the operand
+    // quad of mma.sync (standard fragment layouts; MMA row slot gid is tile row 16*mt + gid) - the 128-bit
+    // loads of the other scheme cost about 29 register moves per 16 x 32 unit to interleave two rows into
+    // quads.  g = 16: the scale arithmetic, not the instruction count, bounds that instantiation and the
+    // longer ldmatrix latency measured slower, so it keeps the permuted contraction index: every lane reads 16
+    // contiguous bytes of its two rows and of a transform row; row slot gid reads tile row 16*mt + pi(gid),
+    // pi = (0,4,1,5,2,6,3,7), so that the two rows of a quarter-warp fall into disjoint bank halves.
+    constexpr bool LDSM = (G == 32);
+    const int prow = LDSM ? 16 * mt + gid : 16 * mt + ((gid & 1) << 2) + (gid >> 1);
     const int sbp = warp >> 3;                // super-blocks 2*sbp, 2*sbp+1 of the panel
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
@@ -158,6 +178,25 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     const int KB32 = (int)KB;
     const int ktiles = (KB32 + 3) >> 2;
     const int64_t code_pitch = K >> 1;
+    // Everything that does not change from item to item is worked out once: the shared-memory addresses of
+    // this lane's two 16-byte pieces per super-block (32-bit, relative to the stage), and the steps by which
+    // the output pointers advance when the row block does.
+    // ldmatrix.x4: lane l addresses row (l & 7) + 8 * ((l >> 3) & 1) of the warp's 16-row slice and the 16-byte
+    // chunk c0 + (l >> 4) of its 128-byte box row; chunk index XORed with (row & 7) by the TMA swizzle
+    const int lm_row = LDSM ? 16 * mt + (lane & 7) + ((lane >> 3) & 1) * 8 : prow;
+    const uint32_t x_base = sq_smem_u32(smem) + sbp * (2 * SQ_SB_BYTES) + lm_row * 128;
+    // (super-block q, k-step ks) -> chunk c = 4q + 2ks (+1 for lanes >= 16), at byte ((c ^ (row & 7)) << 4):
+    // x_sw holds the lane's XOR term, already shifted
+    // (g = 16: the lane's chunks are tig and 4 + tig of its own row, XOR term prow & 7)
+    const uint32_t x_sw = LDSM ? static_cast<uint32_t>(((lane >> 4) ^ (lane & 7)) << 4)
+                               : static_cast<uint32_t>((tig ^ (prow & 7)) << 4);
+    // (the host takes this kernel only while both output buffers stay below 4 GiB: 32-bit byte offsets)
+    const uint32_t code_pitch32 = static_cast<uint32_t>(code_pitch);
+    const uint32_t code_step = SQ_ROWS * code_pitch32;
+    const uint32_t sf_step = (sf_layout == 0) ? SQ_ROWS * KB32 : ktiles * 512;   // SQ_ROWS = one 128-row scale tile
+    const bool m_ragged = (M % SQ_ROWS) != 0;
+    uint32_t code_off = 0;                    // codes of (row rA, this lane's 8 bytes) for the current item
+    uint32_t sf_off = 0;                      // scale bytes of (row rA, first block of this warp's super-block pair)
     for (int it = item_begin; it < item_end; ++it, ++n) {
       const int nsb = min(4, total_sb - panel * 4);
       if (panel != cur_panel) {
@@ -168,17 +207,27 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
             const int r = 8 * nchunk + 2 * t + (gid & 1);     // transform row for column slot gid of tile t
+            // B fragment of column slot gid: channels 2*tig, 2*tig+1 (+8) of k-step 0 in .x (.y), of k-step 1 in .z (.w)
             uint4 w = make_uint4(0, 0, 0, 0);
             if (2 * sbp + q < nsb) {
               if (G == 32) {
-                w = __ldg(reinterpret_cast<const uint4*>(T + ((int64_t)sb * 32 + r) * 32 + 8 * tig));
-              } else if ((r >> 4) == (tig >> 1)) {              // block-diagonal pair: off-diagonal chunks are zero
+                const uint32_t* row = reinterpret_cast<const uint32_t*>(T + ((int64_t)sb * 32 + r) * 32);
+                w = make_uint4(__ldg(row + tig), __ldg(row + 4 + tig), __ldg(row + 8 + tig), __ldg(row + 12 + tig));
+              } else if ((r >> 4) == (tig >> 1)) {
+                // permuted contraction index: the lane's 8 channels 8*tig.. belong to block tig >> 1 of the
+                // block-diagonal pair; off-diagonal pieces are zero
                 w = __ldg(reinterpret_cast<const uint4*>(T + (((int64_t)sb * 2 + (r >> 4)) * 16 + (r & 15)) * 16 + 8 * (tig & 1)));
               }
             }
             tf[q][t] = w;
           }
         }
+        // output pointers of this panel at the current row block
+        const uint32_t rA0 = rb * SQ_ROWS + prow;
+        code_off = rA0 * code_pitch32 + (panel * 64 + sbp * 32 + 8 * tig);
+        const int kb0 = (G == 32) ? panel * 4 + 2 * sbp : panel * 8 + 4 * sbp;
+        if (sf_layout == 0) sf_off = rA0 * KB32 + kb0;
+        else sf_off = (rb * ktiles + (kb0 >> 2)) * 512 + (prow & 31) * 16 + (prow >> 5) * 4 + (kb0 & 3);
       }
       const int s = n % SQ_STAGES;
       const uint32_t ph = (n / SQ_STAGES) & 1;
@@ -186,128 +235,134 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x50000 | n); *abort_flag = 1; }
         break;
       }
-      const uint8_t* tile = smem + s * SQ_STAGE_BYTES;
-      uint4 xa[2], xb[2];
+      uint4 af[2][2];                           // A operand quads: [super-block q][k-step]
+      {
+        const uint32_t a = x_base + s * SQ_STAGE_BYTES;   // box sbp holds this warp's two super-blocks
+        // (2c + hi) ^ r7 = 2c ^ (hi ^ r7): bit 0 of 2c is clear, so + is ^ there and XOR associates
+        if (LDSM) {
+          af[0][0] = sq_ldmatrix_x4(a + ((0u << 4) ^ x_sw)); af[0][1] = sq_ldmatrix_x4(a + ((2u << 4) ^ x_sw));
+          af[1][0] = sq_ldmatrix_x4(a + ((4u << 4) ^ x_sw)); af[1][1] = sq_ldmatrix_x4(a + ((6u << 4) ^ x_sw));
+        } else {
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        // box sbp holds this warp's two super-blocks: rows of 128 bytes, 16-byte chunk index XORed
-        // with (row & 7) by the TMA swizzle; rows prow and prow + 8 share the same XOR term
-        const uint8_t* p = tile + sbp * (2 * SQ_SB_BYTES) + prow * 128 + (((4 * q + tig) ^ (prow & 7)) << 4);
-        xa[q] = *reinterpret_cast<const uint4*>(p);
-        xb[q] = *reinterpret_cast<const uint4*>(p + 8 * 128);
+          for (int q = 0; q < 2; ++q) {         // rows prow and prow + 8 share the XOR term; chunk 4q + tig
+            const uint4 xa = sq_lds128(a + ((4u * q << 4) ^ x_sw)), xb = sq_lds128(a + ((4u * q << 4) ^ x_sw) + 8 * 128);
+            af[q][0] = make_uint4(xa.x, xb.x, xa.y, xb.y);
+            af[q][1] = make_uint4(xa.z, xb.z, xa.w, xb.w);
+          }
+        }
       }
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sq_smem_u32(&empty_bar[s])) : "memory");
 
-      const int this_panel = panel, this_rb = rb;
-      if (++rb == num_rb) { rb = 0; ++panel; }
+      uint8_t* const pa = codes + code_off;
+      uint8_t* const ps = scales + sf_off;
+      const bool last_rb = (rb == num_rb - 1);
+      if (++rb == num_rb) { rb = 0; ++panel; } else { code_off += code_step; sf_off += sf_step; }
       if (2 * sbp >= nsb) continue;             // K tail: this warp's super-blocks do not exist
-      const int rA = this_rb * SQ_ROWS + prow, rB = rA + 8;
-      const bool okA = rA < M, okB = rB < M;
-      uint32_t wA[2], wB[2], sA[2], sB[2];
+
+      // One item: FULL = every row and both super-blocks of this warp exist (no predicates at all).
+      auto item = [&](auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
+        bool okA = true, okB = true;
+        if (!FULL) {
+          const int rA = (last_rb ? (num_rb - 1) : 0) * SQ_ROWS + prow;   // only the last row block can be ragged
+          okA = !last_rb || rA < M;
+          okB = !last_rb || rA + 8 < M;
+        }
+        uint32_t wA[2], wB[2], sA[2], sB[2];
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        float acc[4][4];
+        for (int q = 0; q < 2; ++q) {
+          float acc[4][4];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          mma_bf16_16816_first(acc[t], xa[q].x, xb[q].x, xa[q].y, xb[q].y, tf[q][t].x, tf[q][t].y);
-          mma_bf16_16816(acc[t], xa[q].z, xb[q].z, xa[q].w, xb[q].w, tf[q][t].z, tf[q][t].w);
-        }
-        float vA[8], vB[8];
+          for (int t = 0; t < 4; ++t) {
+            mma_bf16_16816_first(acc[t], af[q][0].x, af[q][0].y, af[q][0].z, af[q][0].w, tf[q][t].x, tf[q][t].y);
+            mma_bf16_16816(acc[t], af[q][1].x, af[q][1].y, af[q][1].z, af[q][1].w, tf[q][t].z, tf[q][t].w);
+          }
+          float vA[8], vB[8];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          vA[2 * t] = acc[t][0]; vA[2 * t + 1] = acc[t][1];
-          vB[2 * t] = acc[t][2]; vB[2 * t + 1] = acc[t][3];
-        }
-        // AbsMax of the lane's 8 values per row as a tree of 3-input maxima (sm_100 has a 3-input FMNMX)
-        float aA = fmaxf(fmaxf(fabsf(vA[0]), fabsf(vA[1])), fabsf(vA[2]));
-        aA = fmaxf(fmaxf(aA, fabsf(vA[3])), fabsf(vA[4]));
-        aA = fmaxf(fmaxf(aA, fabsf(vA[5])), fmaxf(fabsf(vA[6]), fabsf(vA[7])));
-        float aB = fmaxf(fmaxf(fabsf(vB[0]), fabsf(vB[1])), fabsf(vB[2]));
-        aB = fmaxf(fmaxf(aB, fabsf(vB[3])), fabsf(vB[4]));
-        aB = fmaxf(fmaxf(aB, fabsf(vB[5])), fmaxf(fabsf(vB[6]), fabsf(vB[7])));
-        if (AMAX) { seen = fmaxf(seen, fmaxf(okA ? aA : 0.0f, okB ? aB : 0.0f)); continue; }
-        aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 2));       // lanes tig and tig^2 share a g=16 block
-        aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 2));
-        if (G == 32) {
-          aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 1));
-          aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 1));
-        }
-        float mA, mB;
-        if (FMT == kFmtMX) {
-          mx_scale(aA, sA[q], mA, mx_ceil); mx_scale(aB, sB[q], mB, mx_ceil);
-        } else {
-          // four distinct scales per quad (row A/B x block 0/1): lane tig computes the one of
-          // (row tig>>1, its own block) and fetches the other row's from lane tig^2
-          const bool mine_is_b = (tig >> 1) != 0;
-          uint32_t sm; float mm;
-          nv_scale(mine_is_b ? aB : aA, ts, sm, mm);
-          const uint32_t so = __shfl_xor_sync(0xffffffffu, sm, 2);
-          const float mo = __shfl_xor_sync(0xffffffffu, mm, 2);
-          sA[q] = mine_is_b ? so : sm; mA = mine_is_b ? mo : mm;
-          sB[q] = mine_is_b ? sm : so; mB = mine_is_b ? mm : mo;
-        }
-#pragma unroll
-        for (int i = 0; i < 8; i += 2) { mul2_rn(vA[i], vA[i + 1], mA); mul2_rn(vB[i], vB[i + 1], mB); }
-        wA[q] = pack_e2m1x8_fast(vA);
-        wB[q] = pack_e2m1x8_fast(vB);
-      }
-      if (AMAX) continue;
-      // ---- codes: lanes 0,1 gather super-block 0, lanes 2,3 super-block 1 (8 contiguous bytes each)
-      {
-        const bool lo = tig < 2;
-        const uint32_t rcvA = __shfl_xor_sync(0xffffffffu, lo ? wA[1] : wA[0], 2);
-        const uint32_t rcvB = __shfl_xor_sync(0xffffffffu, lo ? wB[1] : wB[0], 2);
-        const uint2 oA = lo ? make_uint2(wA[0], rcvA) : make_uint2(rcvA, wA[1]);
-        const uint2 oB = lo ? make_uint2(wB[0], rcvB) : make_uint2(rcvB, wB[1]);
-        const bool col_ok = (2 * sbp + (tig >> 1)) < nsb;
-        uint8_t* pa = codes + (int64_t)rA * code_pitch + (this_panel * 64 + sbp * 32 + 8 * tig);
-        if (okA && col_ok) *reinterpret_cast<uint2*>(pa) = oA;
-        if (okB && col_ok) *reinterpret_cast<uint2*>(pa + 8 * code_pitch) = oB;
-      }
-      // ---- scale bytes: one 16-bit (g=32) or 32-bit (g=16) store per row by lane tig == 0
-      if (tig == 0) {
-        const int kb = (G == 32) ? this_panel * 4 + 2 * sbp : this_panel * 8 + 4 * sbp;
-        int64_t offA, offB;
-        if (sf_layout == 0) {
-          offA = (int64_t)rA * KB32 + kb;
-          offB = offA + 8 * (int64_t)KB32;
-        } else {
-          // rows rA and rA + 8 lie in the same 32-row group of the same 128-row tile
-          offA = ((int64_t)(rA >> 7) * ktiles + (kb >> 2)) * 512 + (rA & 31) * 16 + ((rA & 127) >> 5) * 4 + (kb & 3);
-          offB = offA + 8 * 16;
-        }
-        const bool pair_ok = 2 * sbp + 1 < nsb;
-        if (G == 32) {
-          const uint32_t outA = sA[0] | (sA[1] << 8), outB = sB[0] | (sB[1] << 8);
-          if (pair_ok) {
-            if (okA) *reinterpret_cast<uint16_t*>(scales + offA) = (uint16_t)outA;
-            if (okB) *reinterpret_cast<uint16_t*>(scales + offB) = (uint16_t)outB;
+          for (int t = 0; t < 4; ++t) {
+            vA[2 * t] = acc[t][0]; vA[2 * t + 1] = acc[t][1];
+            vB[2 * t] = acc[t][2]; vB[2 * t + 1] = acc[t][3];
+          }
+          // AbsMax of the lane's 8 values per row as a tree of 3-input maxima (sm_100 has a 3-input FMNMX)
+          float aA = fmaxf(fmaxf(fabsf(vA[0]), fabsf(vA[1])), fabsf(vA[2]));
+          aA = fmaxf(fmaxf(aA, fabsf(vA[3])), fabsf(vA[4]));
+          aA = fmaxf(fmaxf(aA, fabsf(vA[5])), fmaxf(fabsf(vA[6]), fabsf(vA[7])));
+          float aB = fmaxf(fmaxf(fabsf(vB[0]), fabsf(vB[1])), fabsf(vB[2]));
+          aB = fmaxf(fmaxf(aB, fabsf(vB[3])), fabsf(vB[4]));
+          aB = fmaxf(fmaxf(aB, fabsf(vB[5])), fmaxf(fabsf(vB[6]), fabsf(vB[7])));
+          if (AMAX) { seen = fmaxf(seen, fmaxf(okA ? aA : 0.0f, okB ? aB : 0.0f)); continue; }
+          aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 2));       // lanes tig and tig^2 share a g=16 block
+          aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 2));
+          if (G == 32) {
+            aA = fmaxf(aA, __shfl_xor_sync(0xffffffffu, aA, 1));
+            aB = fmaxf(aB, __shfl_xor_sync(0xffffffffu, aB, 1));
+          }
+          float mA, mB;
+          if (FMT == kFmtMX) {
+            mx_scale(aA, sA[q], mA, mx_ceil); mx_scale(aB, sB[q], mB, mx_ceil);
           } else {
-            if (okA) scales[offA] = (uint8_t)outA;
-            if (okB) scales[offB] = (uint8_t)outB;
+            // four distinct scales per quad (row A/B x block 0/1): lane tig computes the one of
+            // (row tig>>1, its own block) and fetches the other row's from lane tig^2
+            const bool mine_is_b = (tig >> 1) != 0;
+            uint32_t sm; float mm;
+            nv_scale(mine_is_b ? aB : aA, ts, sm, mm);
+            const uint32_t so = __shfl_xor_sync(0xffffffffu, sm, 2);
+            const float mo = __shfl_xor_sync(0xffffffffu, mm, 2);
+            sA[q] = mine_is_b ? so : sm; mA = mine_is_b ? mo : mm;
+            sB[q] = mine_is_b ? sm : so; mB = mine_is_b ? mm : mo;
+          }
+          const uint64_t mA2 = pair_of(mA), mB2 = pair_of(mB);       // {m, m} built once per row
+#pragma unroll
+          for (int i = 0; i < 8; i += 2) { mul2_rn(vA[i], vA[i + 1], mA2); mul2_rn(vB[i], vB[i + 1], mB2); }
+          wA[q] = pack_e2m1x8_fast(vA);
+          wB[q] = pack_e2m1x8_fast(vB);
+        }
+        if (AMAX) return;
+        // ---- codes: lanes 0,1 gather super-block 0, lanes 2,3 super-block 1 (8 contiguous bytes each)
+        {
+          const bool lo = tig < 2;
+          const uint32_t rcvA = __shfl_xor_sync(0xffffffffu, lo ? wA[1] : wA[0], 2);
+          const uint32_t rcvB = __shfl_xor_sync(0xffffffffu, lo ? wB[1] : wB[0], 2);
+          const uint2 oA = lo ? make_uint2(wA[0], rcvA) : make_uint2(rcvA, wA[1]);
+          const uint2 oB = lo ? make_uint2(wB[0], rcvB) : make_uint2(rcvB, wB[1]);
+          const bool col_ok = FULL || (2 * sbp + (tig >> 1)) < nsb;
+          if (okA && col_ok) *reinterpret_cast<uint2*>(pa) = oA;
+          if (okB && col_ok) *reinterpret_cast<uint2*>(pa + 8 * code_pitch32) = oB;
+        }
+        // ---- scale bytes: rows rA and rA + 8 lie in the same 32-row group of the same 128-row tile
+        const uint32_t sf_row8 = (sf_layout == 0) ? 8 * KB32 : 8 * 16;
+        const bool pair_ok = FULL || (2 * sbp + 1 < nsb);
+        if (G == 32) {
+          // one 16-bit store per row by lane tig == 0
+          if (tig == 0) {
+            const uint32_t outA = sA[0] | (sA[1] << 8), outB = sB[0] | (sB[1] << 8);
+            if (pair_ok) {
+              if (okA) *reinterpret_cast<uint16_t*>(ps) = (uint16_t)outA;
+              if (okB) *reinterpret_cast<uint16_t*>(ps + sf_row8) = (uint16_t)outB;
+            } else {
+              if (okA) ps[0] = (uint8_t)outA;
+              if (okB) ps[sf_row8] = (uint8_t)outB;
+            }
+          }
+        } else {
+          // lanes tig 0,2 hold the first block of each super-block, lanes 1,3 the second: one 32-bit store per row
+          const uint32_t mineA = sA[0] | (sA[1] << 16), mineB = sB[0] | (sB[1] << 16);
+          const uint32_t othA = __shfl_xor_sync(0xffffffffu, mineA, 1), othB = __shfl_xor_sync(0xffffffffu, mineB, 1);
+          if (tig == 0) {
+            const uint32_t outA = mineA | (othA << 8), outB = mineB | (othB << 8);
+            if (pair_ok) {
+              if (okA) *reinterpret_cast<uint32_t*>(ps) = outA;
+              if (okB) *reinterpret_cast<uint32_t*>(ps + sf_row8) = outB;
+            } else {
+              if (okA) *reinterpret_cast<uint16_t*>(ps) = (uint16_t)outA;
+              if (okB) *reinterpret_cast<uint16_t*>(ps + sf_row8) = (uint16_t)outB;
+            }
           }
         }
-      }
-      if (G == 16) {
-        // lanes tig 0,2 hold the first block of each super-block, lanes 1,3 the second
-        const uint32_t mineA = sA[0] | (sA[1] << 16), mineB = sB[0] | (sB[1] << 16);
-        const uint32_t othA = __shfl_xor_sync(0xffffffffu, mineA, 1), othB = __shfl_xor_sync(0xffffffffu, mineB, 1);
-        if (tig == 0) {
-          const int kb = this_panel * 8 + 4 * sbp;
-          int64_t offA, offB;
-          if (sf_layout == 0) { offA = (int64_t)rA * KB32 + kb; offB = offA + 8 * (int64_t)KB32; }
-          else { offA = ((int64_t)(rA >> 7) * ktiles + (kb >> 2)) * 512 + (rA & 31) * 16 + ((rA & 127) >> 5) * 4; offB = offA + 8 * 16; }
-          const uint32_t outA = mineA | (othA << 8), outB = mineB | (othB << 8);
-          if (2 * sbp + 1 < nsb) {
-            if (okA) *reinterpret_cast<uint32_t*>(scales + offA) = outA;
-            if (okB) *reinterpret_cast<uint32_t*>(scales + offB) = outB;
-          } else {
-            if (okA) *reinterpret_cast<uint16_t*>(scales + offA) = (uint16_t)outA;
-            if (okB) *reinterpret_cast<uint16_t*>(scales + offB) = (uint16_t)outB;
-          }
-        }
-      }
+      };
+      if (nsb == 4 && !(last_rb && m_ragged)) item(std::true_type());
+      else item(std::false_type());
     }
     if (AMAX) {
 #pragma unroll
@@ -368,6 +423,7 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   const int64_t panels = (K / 32 + 3) / 4;
   const int64_t items = panels * num_rb;
   if (items > 0x7fffffff || M > 0x7fffff00) return cudaErrorNotSupported;
+  if ((M + SQ_ROWS) * (K / 2) >= ((int64_t)1 << 32)) return cudaErrorNotSupported;   // the kernel keeps 32-bit output offsets
   const int grid = (int)(items < sm_count ? items : sm_count);
   const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
   const int cs = clear_status ? 1 : 0;

@@ -51,6 +51,21 @@ __device__ __forceinline__ uint32_t pack_e2m1x8_fast(const float (&u)[8]) {
   return w;
 }
 
+// the register pair {m, m}: second operand of the packed multiply below
+__device__ __forceinline__ uint64_t pair_of(float m) {
+  uint64_t p;
+  asm("mov.b64 %0, {%1, %1};" : "=l"(p) : "f"(m));
+  return p;
+}
+// (a, b) * (m, m) with one packed fp32 instruction (round to nearest, no flush), multiplier given as pair_of(m)
+__device__ __forceinline__ void mul2_rn(float& a, float& b, uint64_t mm) {
+  asm("{\n\t.reg .b64 v;\n\t"
+      "mov.b64 v, {%0, %1};\n\t"
+      "mul.rn.f32x2 v, v, %2;\n\t"
+      "mov.b64 {%0, %1}, v;\n\t}"
+      : "+f"(a), "+f"(b)
+      : "l"(mm));
+}
 // (a, b) * (m, m) with one packed fp32 instruction (round to nearest, no flush)
 __device__ __forceinline__ void mul2_rn(float& a, float& b, float m) {
   asm("{\n\t.reg .b64 v, s;\n\t"
