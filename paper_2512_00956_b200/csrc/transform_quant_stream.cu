@@ -29,7 +29,7 @@ constexpr int SQ_CONSUMERS = 16;
 constexpr int SQ_THREADS = (SQ_CONSUMERS + 1) * 32;
 constexpr int SQ_SB_BYTES = SQ_ROWS * 64;              // one super-block of a tile: 128 rows x 64 B
 constexpr int SQ_STAGE_BYTES = 4 * SQ_SB_BYTES;        // 32 KiB
-constexpr int SQ_SMEM = SQ_STAGES * SQ_STAGE_BYTES + 1024 + 128;
+constexpr int SQ_SMEM = SQ_STAGES * SQ_STAGE_BYTES + 1024 + 128 + 512;   // ring, alignment slack, barriers, NVFP4 multiplier table
 
 __device__ __forceinline__ uint32_t sq_smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ bool sq_try_wait(uint32_t bar, uint32_t parity) {
@@ -84,6 +84,15 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
   uint64_t* empty_bar = full_bar + SQ_STAGES;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + SQ_STAGES);
 
+  // NVFP4: 1 / (float(scale byte) * ts) for all 128 scale bytes, the same two roundings as nv_scale, done once
+  float* nv_mult = reinterpret_cast<float*>(smem + SQ_STAGES * SQ_STAGE_BYTES + 128);
+  const bool nv_quant = (FMT == kFmtNV) && !AMAX;
+  const bool nv_dynamic = nv_quant && amax_in != nullptr;
+  float ts = 1.0f;
+  if (nv_quant && !nv_dynamic) {              // static scale: a calibration constant, not the previous kernel's output
+    ts = *ts_ptr;
+    if (threadIdx.x < 128) nv_mult[threadIdx.x] = nv_mult_of_byte(threadIdx.x, ts);
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 32) prefetch_tensormap(&mapX);
   if (threadIdx.x == 0) {
@@ -101,6 +110,12 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
   // the status word is only ever set after a bounded wait of about a second has expired, so clearing it
   // here cannot race with a report; it saves wush_linear a separate memset between kernels
   if (clear_status && blockIdx.x == 0 && threadIdx.x == 0 && status != nullptr) *status = 0;
+  if (nv_dynamic) {                           // per-batch tensor scale from the AbsMax pass that ran before
+    ts = nv_tensor_scale(__uint_as_float(*amax_in));
+    if (threadIdx.x < 128) nv_mult[threadIdx.x] = nv_mult_of_byte(threadIdx.x, ts);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && ts_out != nullptr) *ts_out = ts;
+    __syncthreads();
+  }
   // let a programmatic dependent (the GEMM of wush_linear) be scheduled as SMs free up; it still waits
   // for this whole grid before reading the codes
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -160,16 +175,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     const int sbp = warp >> 3;                // super-blocks 2*sbp, 2*sbp+1 of the panel
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
-    float ts = 1.0f;
     float seen = 0.0f;                         // AMAX: running maximum of this lane
-    if (FMT == kFmtNV && !AMAX) {
-      if (amax_in != nullptr) {                 // per-batch tensor scale from the AbsMax pass that ran before
-        ts = nv_tensor_scale(__uint_as_float(*amax_in));
-        if (blockIdx.x == 0 && threadIdx.x == 0 && ts_out != nullptr) *ts_out = ts;
-      } else {
-        ts = *ts_ptr;
-      }
-    }
 
     uint4 tf[2][4];                           // B fragments of the two transforms, kept across items
     int cur_panel = -1;
@@ -305,12 +311,10 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
             // four distinct scales per quad (row A/B x block 0/1): lane tig computes the one of
             // (row tig>>1, its own block) and fetches the other row's from lane tig^2
             const bool mine_is_b = (tig >> 1) != 0;
-            uint32_t sm; float mm;
-            nv_scale(mine_is_b ? aB : aA, ts, sm, mm);
+            const uint32_t sm = nv_scale_byte(mine_is_b ? aB : aA, ts);
             const uint32_t so = __shfl_xor_sync(0xffffffffu, sm, 2);
-            const float mo = __shfl_xor_sync(0xffffffffu, mm, 2);
-            sA[q] = mine_is_b ? so : sm; mA = mine_is_b ? mo : mm;
-            sB[q] = mine_is_b ? sm : so; mB = mine_is_b ? mm : mo;
+            sA[q] = mine_is_b ? so : sm; mA = nv_mult[sA[q]];
+            sB[q] = mine_is_b ? sm : so; mB = nv_mult[sB[q]];
           }
           const uint64_t mA2 = pair_of(mA), mB2 = pair_of(mB);       // {m, m} built once per row
 #pragma unroll

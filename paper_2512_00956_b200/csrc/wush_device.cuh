@@ -104,11 +104,19 @@ __device__ __forceinline__ float nv_tensor_scale(float amax) {
 
 // ---- NVFP4 scale.  Single-rounded fp32 steps, in this order and with no contraction:
 //   r = (amax / 6) / ts ;  byte = E4M3(r) ;  d = float(byte) * ts ;  mult = d == 0 ? 0 : 1 / d.
-__device__ __forceinline__ void nv_scale(float amax, float ts, uint32_t& byte, float& mult) {
+// The two halves separately: the scale byte of a block, and the multiplier that belongs to a scale byte.
+// The multiplier depends on (byte, ts) only, so a kernel may tabulate it for the 128 byte values once.
+__device__ __forceinline__ uint32_t nv_scale_byte(float amax, float ts) {
   const float r = __fdiv_rn(__fdiv_rn(amax, 6.0f), ts);
-  byte = static_cast<uint32_t>(__nv_cvt_float_to_fp8(r, __NV_SATFINITE, __NV_E4M3));
+  return static_cast<uint32_t>(__nv_cvt_float_to_fp8(r, __NV_SATFINITE, __NV_E4M3));
+}
+__device__ __forceinline__ float nv_mult_of_byte(uint32_t byte, float ts) {
   const float d = __fmul_rn(e4m3_to_float(byte), ts);
-  mult = (d == 0.0f) ? 0.0f : __frcp_rn(d);
+  return (d == 0.0f) ? 0.0f : __frcp_rn(d);
+}
+__device__ __forceinline__ void nv_scale(float amax, float ts, uint32_t& byte, float& mult) {
+  byte = nv_scale_byte(amax, ts);
+  mult = nv_mult_of_byte(byte, ts);
 }
 
 // D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
