@@ -3,17 +3,21 @@
 // busy.
 //
 //  * Persistent CTAs (one per SM): 1 producer warp + 16 consumer warps.  The producer streams
-//    128-row x 128-channel tiles of X into a 4-stage shared-memory ring with TMA (two
-//    128-byte-wide boxes per tile, 128-byte swizzle, no multicast), so up to 96 KB per SM are in
-//    flight without costing a register.
-//  * A work item is (128-channel panel, 128-row block); a CTA takes a contiguous run of items in
+//    ROWS-row x 128-channel tiles of X into a shared-memory ring of 128 KB with TMA (two
+//    128-byte-wide boxes per tile, 128-byte swizzle, no multicast): 4 stages of 128 rows, or, for
+//    small problems, 8 stages of 64 rows - finer work items, so the first one lands sooner and the
+//    CTAs finish closer together.
+//  * A work item is (128-channel panel, ROWS-row block); a CTA takes a contiguous run of items in
 //    panel-major order, so the panel rarely changes.  Each consumer warp owns one 16-row slice
-//    and two of the panel's four 32-channel super-blocks, and keeps the MMA B-fragments of those
-//    two transforms in REGISTERS for as long as the panel stays the same (32 registers): in
-//    steady state the only loads are two 128-bit shared-memory reads per super-block.
+//    and two (ROWS = 128) or one (ROWS = 64) of the panel's four 32-channel super-blocks, and keeps
+//    the MMA B-fragments of those transforms in REGISTERS for as long as the panel stays the same.
+//  * A operands: g = 32 uses ldmatrix.x4 (its destination registers are the MMA operand quad);
+//    g = 16 reads 16 contiguous bytes per lane and row with a permuted contraction index.
 //  * Output permutation: MMA column slot (tile t, n) carries transform row 8*c(n/2) + 2*t + n%2
-//    with c = (0,2,1,3), so after one shuffle with lane^2 every lane owns 8 contiguous code
-//    bytes and a row's 32 bytes leave as one full sector per quad.
+//    with c = (0,2,1,3), so every lane owns 8 consecutive outputs = 4 code bytes; with two
+//    super-blocks per warp one shuffle with lane^2 makes that 8 contiguous bytes and a row's 32
+//    bytes leave as one full sector per quad.
+//  * Interior items (all rows and super-blocks present) run a copy of the item body without predicates.
 #include <cuda.h>
 
 #include <type_traits>
@@ -23,13 +27,17 @@
 
 namespace wush {
 
-constexpr int SQ_ROWS = 128;
-constexpr int SQ_STAGES = 4;
+// Tile geometry.  ROWS = 128: 16 warps = 8 row slices x 2 pairs of super-blocks, 4 ring stages of 32 KB.
+// ROWS = 64 (small problems: finer work items, the first one lands sooner, CTAs end closer together):
+// 16 warps = 4 row slices x 4 super-blocks, 8 stages of 16 KB.  Bytes in flight are the same.
+constexpr int SQ_RING_BYTES = 128 * 1024;
+constexpr int SQ_MAX_STAGES = 8;
+constexpr int SQ_SMALL = 5;          // fewer 128-row items per CTA than this: use 64-row tiles (measured: 3.5 per
+                                     // CTA gains 7-25 %, 7 per CTA loses 6 %, large problems are unchanged)
 constexpr int SQ_CONSUMERS = 16;
 constexpr int SQ_THREADS = (SQ_CONSUMERS + 1) * 32;
-constexpr int SQ_SB_BYTES = SQ_ROWS * 64;              // one super-block of a tile: 128 rows x 64 B
-constexpr int SQ_STAGE_BYTES = 4 * SQ_SB_BYTES;        // 32 KiB
-constexpr int SQ_SMEM = SQ_STAGES * SQ_STAGE_BYTES + 1024 + 128 + 512;   // ring, alignment slack, barriers, NVFP4 multiplier table
+// ring | full[8] empty[8] barriers (128 B) | abort flag (64 B) | NVFP4 multiplier table (512 B); 1 KiB alignment slack
+constexpr int SQ_SMEM = SQ_RING_BYTES + 1024 + 128 + 64 + 512;
 
 __device__ __forceinline__ uint32_t sq_smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ bool sq_try_wait(uint32_t bar, uint32_t parity) {
@@ -71,21 +79,27 @@ __device__ __forceinline__ bool sq_elect() {
 // AMAX = true: the same tile walk and the same products, but instead of quantising, the AbsMax of everything
 // computed is folded into *ts_out (read as the uint32 bit pattern of a non-negative float, atomicMax): the
 // first pass of the per-batch NVFP4 tensor scale.  codes / scales are not touched.
-template <int G, bool AMAX = false>
+template <int G, bool AMAX = false, int ROWS = 128>
 __global__ void __launch_bounds__(SQ_THREADS, 1)
 tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
                  const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
                  int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status, int clear_status,
                  const uint32_t* __restrict__ amax_in, float* __restrict__ ts_out, int mx_ceil) {
   constexpr int FMT = (G == 32) ? kFmtMX : kFmtNV;
+  constexpr int SQ_ROWS = ROWS;
+  constexpr int NQ = ROWS / 64;                      // super-blocks per consumer warp
+  constexpr int SLICES = ROWS / 16;                  // 16-row slices per tile
+  constexpr int SQ_BOX_BYTES = ROWS * 128;           // one TMA box: ROWS rows x 64 channels
+  constexpr int SQ_STAGE_BYTES = 2 * SQ_BOX_BYTES;   // a 128-channel panel
+  constexpr int SQ_STAGES = SQ_RING_BYTES / SQ_STAGE_BYTES;
   extern __shared__ uint8_t sq_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(sq_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SQ_STAGES * SQ_STAGE_BYTES);
-  uint64_t* empty_bar = full_bar + SQ_STAGES;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + SQ_STAGES);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SQ_RING_BYTES);
+  uint64_t* empty_bar = full_bar + SQ_MAX_STAGES;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + SQ_MAX_STAGES);
 
   // NVFP4: 1 / (float(scale byte) * ts) for all 128 scale bytes, the same two roundings as nv_scale, done once
-  float* nv_mult = reinterpret_cast<float*>(smem + SQ_STAGES * SQ_STAGE_BYTES + 128);
+  float* nv_mult = reinterpret_cast<float*>(smem + SQ_RING_BYTES + 128 + 64);
   const bool nv_quant = (FMT == kFmtNV) && !AMAX;
   const bool nv_dynamic = nv_quant && amax_in != nullptr;
   float ts = 1.0f;
@@ -140,9 +154,9 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
       if (sq_elect()) {
         const uint32_t bar = sq_smem_u32(&full_bar[s]);
         const int nbox = nsb >> 1;                       // 64-channel (128-byte) boxes; K % 64 == 0
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(nbox * 2 * SQ_SB_BYTES) : "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(nbox * SQ_BOX_BYTES) : "memory");
         for (int bx = 0; bx < nbox; ++bx) {
-          const uint32_t dst = sq_smem_u32(smem + s * SQ_STAGE_BYTES + bx * 2 * SQ_SB_BYTES);
+          const uint32_t dst = sq_smem_u32(smem + s * SQ_STAGE_BYTES + bx * SQ_BOX_BYTES);
           asm volatile(
               "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
               ::"r"(dst), "l"(&mapX), "r"((panel * 2 + bx) * 64), "r"(rb * SQ_ROWS), "r"(bar) : "memory");
@@ -162,7 +176,8 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
   } else {
     // ------------------------------------------------------------------ consumer warps
     const int gid = lane >> 2, tig = lane & 3;
-    const int mt = warp & 7;                  // 16-row slice of the tile
+    const int mt = warp % SLICES;             // 16-row slice of the tile
+    const int wsb = (warp / SLICES) * NQ;     // first of this warp's NQ super-blocks (of the panel's four)
     // Two ways to fetch the A operands.  g = 32: ldmatrix, whose four destination registers ARE the operand
     // quad of mma.sync (standard fragment layouts; MMA row slot gid is tile row 16*mt + gid) - the 128-bit
     // loads of the other scheme cost about 29 register moves per 16 x 32 unit to interleave two rows into
@@ -172,12 +187,11 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     // pi = (0,4,1,5,2,6,3,7), so that the two rows of a quarter-warp fall into disjoint bank halves.
     constexpr bool LDSM = (G == 32);
     const int prow = LDSM ? 16 * mt + gid : 16 * mt + ((gid & 1) << 2) + (gid >> 1);
-    const int sbp = warp >> 3;                // super-blocks 2*sbp, 2*sbp+1 of the panel
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
     float seen = 0.0f;                         // AMAX: running maximum of this lane
 
-    uint4 tf[2][4];                           // B fragments of the two transforms, kept across items
+    uint4 tf[NQ][4];                          // B fragments of this warp's transforms, kept across items
     int cur_panel = -1;
     int n = 0;
     int panel = item_begin / num_rb, rb = item_begin % num_rb;
@@ -190,7 +204,8 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     // ldmatrix.x4: lane l addresses row (l & 7) + 8 * ((l >> 3) & 1) of the warp's 16-row slice and the 16-byte
     // chunk c0 + (l >> 4) of its 128-byte box row; chunk index XORed with (row & 7) by the TMA swizzle
     const int lm_row = LDSM ? 16 * mt + (lane & 7) + ((lane >> 3) & 1) * 8 : prow;
-    const uint32_t x_base = sq_smem_u32(smem) + sbp * (2 * SQ_SB_BYTES) + lm_row * 128;
+    const uint32_t x_base = sq_smem_u32(smem) + (wsb >> 1) * SQ_BOX_BYTES + lm_row * 128;   // box wsb / 2
+    const uint32_t x_cb = static_cast<uint32_t>((4 * (wsb & 1)) << 4);                       // first chunk of super-block wsb in its box row
     // (super-block q, k-step ks) -> chunk c = 4q + 2ks (+1 for lanes >= 16), at byte ((c ^ (row & 7)) << 4):
     // x_sw holds the lane's XOR term, already shifted
     // (g = 16: the lane's chunks are tig and 4 + tig of its own row, XOR term prow & 7)
@@ -199,23 +214,21 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     // (the host takes this kernel only while both output buffers stay below 4 GiB: 32-bit byte offsets)
     const uint32_t code_pitch32 = static_cast<uint32_t>(code_pitch);
     const uint32_t code_step = SQ_ROWS * code_pitch32;
-    const uint32_t sf_step = (sf_layout == 0) ? SQ_ROWS * KB32 : ktiles * 512;   // SQ_ROWS = one 128-row scale tile
     const bool m_ragged = (M % SQ_ROWS) != 0;
     uint32_t code_off = 0;                    // codes of (row rA, this lane's 8 bytes) for the current item
-    uint32_t sf_off = 0;                      // scale bytes of (row rA, first block of this warp's super-block pair)
     for (int it = item_begin; it < item_end; ++it, ++n) {
       const int nsb = min(4, total_sb - panel * 4);
       if (panel != cur_panel) {
         cur_panel = panel;
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          const int sb = panel * 4 + 2 * sbp + q;
+        for (int q = 0; q < NQ; ++q) {
+          const int sb = panel * 4 + wsb + q;
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
             const int r = 8 * nchunk + 2 * t + (gid & 1);     // transform row for column slot gid of tile t
             // B fragment of column slot gid: channels 2*tig, 2*tig+1 (+8) of k-step 0 in .x (.y), of k-step 1 in .z (.w)
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (2 * sbp + q < nsb) {
+            if (wsb + q < nsb) {
               if (G == 32) {
                 const uint32_t* row = reinterpret_cast<const uint32_t*>(T + ((int64_t)sb * 32 + r) * 32);
                 w = make_uint4(__ldg(row + tig), __ldg(row + 4 + tig), __ldg(row + 8 + tig), __ldg(row + 12 + tig));
@@ -230,10 +243,9 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         }
         // output pointers of this panel at the current row block
         const uint32_t rA0 = rb * SQ_ROWS + prow;
-        code_off = rA0 * code_pitch32 + (panel * 64 + sbp * 32 + 8 * tig);
-        const int kb0 = (G == 32) ? panel * 4 + 2 * sbp : panel * 8 + 4 * sbp;
-        if (sf_layout == 0) sf_off = rA0 * KB32 + kb0;
-        else sf_off = (rb * ktiles + (kb0 >> 2)) * 512 + (prow & 31) * 16 + (prow >> 5) * 4 + (kb0 & 3);
+        // NQ = 2: after the exchange below lane tig owns bytes 8 tig .. 8 tig + 7 of the pair's 32;  NQ = 1: the
+        // lane's 8 outputs are transform rows 8 c .. 8 c + 7, c = (0,2,1,3)[tig], i.e. bytes 4 c .. 4 c + 3 of 16
+        code_off = rA0 * code_pitch32 + (panel * 64 + wsb * 16 + (NQ == 2 ? 8 * tig : 4 * (((tig & 1) << 1) | (tig >> 1))));
       }
       const int s = n % SQ_STAGES;
       const uint32_t ph = (n / SQ_STAGES) & 1;
@@ -241,17 +253,20 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
         if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x50000 | n); *abort_flag = 1; }
         break;
       }
-      uint4 af[2][2];                           // A operand quads: [super-block q][k-step]
+      uint4 af[NQ][2];                          // A operand quads: [super-block q][k-step]
       {
-        const uint32_t a = x_base + s * SQ_STAGE_BYTES;   // box sbp holds this warp's two super-blocks
-        // (2c + hi) ^ r7 = 2c ^ (hi ^ r7): bit 0 of 2c is clear, so + is ^ there and XOR associates
-        if (LDSM) {
-          af[0][0] = sq_ldmatrix_x4(a + ((0u << 4) ^ x_sw)); af[0][1] = sq_ldmatrix_x4(a + ((2u << 4) ^ x_sw));
-          af[1][0] = sq_ldmatrix_x4(a + ((4u << 4) ^ x_sw)); af[1][1] = sq_ldmatrix_x4(a + ((6u << 4) ^ x_sw));
-        } else {
+        const uint32_t a = x_base + s * SQ_STAGE_BYTES;
+        // chunk index c of a box row sits at byte ((c ^ (row & 7)) << 4).  The chunk bases used here are even
+        // (or multiples of 4) and the lane's own term (lane >> 4, or tig) only touches the bits below, so
+        // (base + term) ^ r7 = base ^ (term ^ r7): XOR the shifted base with the lane's precomputed x_sw
 #pragma unroll
-          for (int q = 0; q < 2; ++q) {         // rows prow and prow + 8 share the XOR term; chunk 4q + tig
-            const uint4 xa = sq_lds128(a + ((4u * q << 4) ^ x_sw)), xb = sq_lds128(a + ((4u * q << 4) ^ x_sw) + 8 * 128);
+        for (int q = 0; q < NQ; ++q) {          // super-block wsb + q starts at chunk x_cb / 16 + 4 q of its box row
+          const uint32_t cb = x_cb + ((4u * q) << 4);
+          if (LDSM) {
+            af[q][0] = sq_ldmatrix_x4(a + (cb ^ x_sw));
+            af[q][1] = sq_ldmatrix_x4(a + ((cb + (2u << 4)) ^ x_sw));
+          } else {                              // rows prow and prow + 8 share the XOR term; the lane's chunk is cb / 16 + tig
+            const uint4 xa = sq_lds128(a + (cb ^ x_sw)), xb = sq_lds128(a + (cb ^ x_sw) + 8 * 128);
             af[q][0] = make_uint4(xa.x, xb.x, xa.y, xb.y);
             af[q][1] = make_uint4(xa.z, xb.z, xa.w, xb.w);
           }
@@ -261,23 +276,30 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sq_smem_u32(&empty_bar[s])) : "memory");
 
       uint8_t* const pa = codes + code_off;
-      uint8_t* const ps = scales + sf_off;
+      uint8_t* ps;                              // scale byte of (row rA, first block of this warp's first super-block)
+      {
+        const uint32_t rA0 = rb * SQ_ROWS + prow;
+        const int kb0 = (G == 32) ? cur_panel * 4 + wsb : cur_panel * 8 + 2 * wsb;
+        if (sf_layout == 0) ps = scales + (rA0 * KB32 + kb0);
+        else ps = scales + (((rA0 >> 7) * ktiles + (kb0 >> 2)) * 512 + (rA0 & 31) * 16 + ((rA0 & 127) >> 5) * 4 + (kb0 & 3));
+      }
+      const int this_rb = rb;
       const bool last_rb = (rb == num_rb - 1);
-      if (++rb == num_rb) { rb = 0; ++panel; } else { code_off += code_step; sf_off += sf_step; }
-      if (2 * sbp >= nsb) continue;             // K tail: this warp's super-blocks do not exist
+      if (++rb == num_rb) { rb = 0; ++panel; } else { code_off += code_step; }
+      if (wsb >= nsb) continue;                 // K tail: this warp's super-blocks do not exist
 
       // One item: FULL = every row and both super-blocks of this warp exist (no predicates at all).
       auto item = [&](auto full_tag) {
         constexpr bool FULL = decltype(full_tag)::value;
         bool okA = true, okB = true;
         if (!FULL) {
-          const int rA = (last_rb ? (num_rb - 1) : 0) * SQ_ROWS + prow;   // only the last row block can be ragged
+          const int rA = this_rb * SQ_ROWS + prow;                       // only the last row block can be ragged
           okA = !last_rb || rA < M;
           okB = !last_rb || rA + 8 < M;
         }
-        uint32_t wA[2], wB[2], sA[2], sB[2];
+        uint32_t wA[NQ], wB[NQ], sA[NQ], sB[NQ];
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
+        for (int q = 0; q < NQ; ++q) {
           float acc[4][4];
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
@@ -323,44 +345,59 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
           wB[q] = pack_e2m1x8_fast(vB);
         }
         if (AMAX) return;
-        // ---- codes: lanes 0,1 gather super-block 0, lanes 2,3 super-block 1 (8 contiguous bytes each)
-        {
+        const uint32_t sf_row8 = (sf_layout == 0) ? 8 * KB32 : 8 * 16;   // rows rA and rA + 8: same 32-row group of a scale tile
+        if (NQ == 2) {
+          // ---- codes: lanes 0,1 gather super-block 0, lanes 2,3 super-block 1 (8 contiguous bytes each)
           const bool lo = tig < 2;
-          const uint32_t rcvA = __shfl_xor_sync(0xffffffffu, lo ? wA[1] : wA[0], 2);
-          const uint32_t rcvB = __shfl_xor_sync(0xffffffffu, lo ? wB[1] : wB[0], 2);
-          const uint2 oA = lo ? make_uint2(wA[0], rcvA) : make_uint2(rcvA, wA[1]);
-          const uint2 oB = lo ? make_uint2(wB[0], rcvB) : make_uint2(rcvB, wB[1]);
-          const bool col_ok = FULL || (2 * sbp + (tig >> 1)) < nsb;
+          const uint32_t rcvA = __shfl_xor_sync(0xffffffffu, lo ? wA[NQ - 1] : wA[0], 2);
+          const uint32_t rcvB = __shfl_xor_sync(0xffffffffu, lo ? wB[NQ - 1] : wB[0], 2);
+          const uint2 oA = lo ? make_uint2(wA[0], rcvA) : make_uint2(rcvA, wA[NQ - 1]);
+          const uint2 oB = lo ? make_uint2(wB[0], rcvB) : make_uint2(rcvB, wB[NQ - 1]);
+          const bool col_ok = FULL || (wsb + (tig >> 1)) < nsb;
           if (okA && col_ok) *reinterpret_cast<uint2*>(pa) = oA;
           if (okB && col_ok) *reinterpret_cast<uint2*>(pa + 8 * code_pitch32) = oB;
-        }
-        // ---- scale bytes: rows rA and rA + 8 lie in the same 32-row group of the same 128-row tile
-        const uint32_t sf_row8 = (sf_layout == 0) ? 8 * KB32 : 8 * 16;
-        const bool pair_ok = FULL || (2 * sbp + 1 < nsb);
-        if (G == 32) {
-          // one 16-bit store per row by lane tig == 0
-          if (tig == 0) {
-            const uint32_t outA = sA[0] | (sA[1] << 8), outB = sB[0] | (sB[1] << 8);
-            if (pair_ok) {
-              if (okA) *reinterpret_cast<uint16_t*>(ps) = (uint16_t)outA;
-              if (okB) *reinterpret_cast<uint16_t*>(ps + sf_row8) = (uint16_t)outB;
-            } else {
-              if (okA) ps[0] = (uint8_t)outA;
-              if (okB) ps[sf_row8] = (uint8_t)outB;
+          // ---- scale bytes of the pair of super-blocks
+          const bool pair_ok = FULL || (wsb + 1 < nsb);
+          if (G == 32) {
+            if (tig == 0) {                      // one 16-bit store per row
+              const uint32_t outA = sA[0] | (sA[NQ - 1] << 8), outB = sB[0] | (sB[NQ - 1] << 8);
+              if (pair_ok) {
+                if (okA) *reinterpret_cast<uint16_t*>(ps) = (uint16_t)outA;
+                if (okB) *reinterpret_cast<uint16_t*>(ps + sf_row8) = (uint16_t)outB;
+              } else {
+                if (okA) ps[0] = (uint8_t)outA;
+                if (okB) ps[sf_row8] = (uint8_t)outB;
+              }
+            }
+          } else {
+            // lanes tig 0,2 hold the first block of each super-block, lanes 1,3 the second: one 32-bit store per row
+            const uint32_t mineA = sA[0] | (sA[NQ - 1] << 16), mineB = sB[0] | (sB[NQ - 1] << 16);
+            const uint32_t othA = __shfl_xor_sync(0xffffffffu, mineA, 1), othB = __shfl_xor_sync(0xffffffffu, mineB, 1);
+            if (tig == 0) {
+              const uint32_t outA = mineA | (othA << 8), outB = mineB | (othB << 8);
+              if (pair_ok) {
+                if (okA) *reinterpret_cast<uint32_t*>(ps) = outA;
+                if (okB) *reinterpret_cast<uint32_t*>(ps + sf_row8) = outB;
+              } else {
+                if (okA) *reinterpret_cast<uint16_t*>(ps) = (uint16_t)outA;
+                if (okB) *reinterpret_cast<uint16_t*>(ps + sf_row8) = (uint16_t)outB;
+              }
             }
           }
         } else {
-          // lanes tig 0,2 hold the first block of each super-block, lanes 1,3 the second: one 32-bit store per row
-          const uint32_t mineA = sA[0] | (sA[1] << 16), mineB = sB[0] | (sB[1] << 16);
-          const uint32_t othA = __shfl_xor_sync(0xffffffffu, mineA, 1), othB = __shfl_xor_sync(0xffffffffu, mineB, 1);
-          if (tig == 0) {
-            const uint32_t outA = mineA | (othA << 8), outB = mineB | (othB << 8);
-            if (pair_ok) {
-              if (okA) *reinterpret_cast<uint32_t*>(ps) = outA;
-              if (okB) *reinterpret_cast<uint32_t*>(ps + sf_row8) = outB;
-            } else {
-              if (okA) *reinterpret_cast<uint16_t*>(ps) = (uint16_t)outA;
-              if (okB) *reinterpret_cast<uint16_t*>(ps + sf_row8) = (uint16_t)outB;
+          // ---- one super-block per warp: every lane stores its own 4 code bytes (a quad covers the 16 bytes)
+          if (okA) *reinterpret_cast<uint32_t*>(pa) = wA[0];
+          if (okB) *reinterpret_cast<uint32_t*>(pa + 8 * code_pitch32) = wB[0];
+          if (G == 32) {
+            if (tig == 0) {
+              if (okA) ps[0] = (uint8_t)sA[0];
+              if (okB) ps[sf_row8] = (uint8_t)sB[0];
+            }
+          } else {                               // the super-block's two block scales: lanes tig 0 and 1
+            const uint32_t othA = __shfl_xor_sync(0xffffffffu, sA[0], 1), othB = __shfl_xor_sync(0xffffffffu, sB[0], 1);
+            if (tig == 0) {
+              if (okA) *reinterpret_cast<uint16_t*>(ps) = (uint16_t)(sA[0] | (othA << 8));
+              if (okB) *reinterpret_cast<uint16_t*>(ps + sf_row8) = (uint16_t)(sB[0] | (othB << 8));
             }
           }
         }
@@ -394,40 +431,34 @@ static SqEncodeFn sq_encode_fn() {
   return fn;
 }
 
-// Returns cudaErrorNotSupported when the streaming kernel cannot take the problem (the caller
-// then uses the register-staged kernel).
-cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
-                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl,
-                                    cudaStream_t st, const QuantOpts& opt) {
+// One launch for a given tile height.  cudaErrorNotSupported: use the register-staged kernel instead.
+template <int ROWS>
+static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
+                                 uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl,
+                                 cudaStream_t st, const QuantOpts& opt, int sm_count) {
   SqEncodeFn enc = sq_encode_fn();
-  if (!enc) return cudaErrorNotSupported;
-  if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
   CUtensorMap map;
   const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
   const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)SQ_ROWS};
+  const cuuint32_t box[2] = {64, (cuuint32_t)ROWS};
   const cuuint32_t estr[2] = {1, 1};
   if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorNotSupported;
-  static int sm_count = 0;
   static bool attr_done = false;
   cudaError_t e;
   if (!attr_done) {
-    int dev = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(tq_stream_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<32, false, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, false, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, true, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
     attr_done = true;
   }
-  const int num_rb = (int)((M + SQ_ROWS - 1) / SQ_ROWS);
+  const int num_rb = (int)((M + ROWS - 1) / ROWS);
   const int64_t panels = (K / 32 + 3) / 4;
   const int64_t items = panels * num_rb;
   if (items > 0x7fffffff || M > 0x7fffff00) return cudaErrorNotSupported;
-  if ((M + SQ_ROWS) * (K / 2) >= ((int64_t)1 << 32)) return cudaErrorNotSupported;   // the kernel keeps 32-bit output offsets
+  if ((M + ROWS) * (K / 2) >= ((int64_t)1 << 32)) return cudaErrorNotSupported;   // the kernel keeps 32-bit output offsets
   const int grid = (int)(items < sm_count ? items : sm_count);
   const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
   const int cs = clear_status ? 1 : 0;
@@ -437,15 +468,15 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   const int mx_ceil = opt.mx_ceil ? 1 : 0;
   if (opt.amax_out != nullptr) {                 // AbsMax pass only (g = 16)
     if (g != 16) return cudaErrorNotSupported;
-    tq_stream_kernel<16, true><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, nullptr, nullptr, nullptr, sf, num_rb, n_items,
-                                                                  nullptr, 0, nullptr, reinterpret_cast<float*>(opt.amax_out), 0);
+    tq_stream_kernel<16, true, ROWS><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, nullptr, nullptr, nullptr, sf, num_rb, n_items,
+                                                                        nullptr, 0, nullptr, reinterpret_cast<float*>(opt.amax_out), 0);
     return cudaGetLastError();
   }
   if (!pdl) {
     if (g == 32)
-      tq_stream_kernel<32><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+      tq_stream_kernel<32, false, ROWS><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
     else
-      tq_stream_kernel<16><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+      tq_stream_kernel<16, false, ROWS><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
     return cudaGetLastError();
   }
   // programmatic dependent launch: set-up overlaps the tail of the previous kernel of the stream
@@ -460,8 +491,30 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (g == 32)
-    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
-  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32, false, ROWS>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16, false, ROWS>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+}
+
+// Returns cudaErrorNotSupported when the streaming kernel cannot take the problem (the caller
+// then uses the register-staged kernel).
+cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
+                                    uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl,
+                                    cudaStream_t st, const QuantOpts& opt) {
+  if (!sq_encode_fn()) return cudaErrorNotSupported;
+  if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0;
+    cudaError_t e;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  }
+  // 128-row tiles unless the problem is small: with fewer than SQ_SMALL of them per CTA the 64-row tiles'
+  // finer items win (the first tile lands sooner and the CTAs finish closer together)
+  const int64_t items128 = ((K / 32 + 3) / 4) * ((M + 127) / 128);
+  if (items128 < (int64_t)SQ_SMALL * sm_count)
+    return launch_stream<64>(X, M, K, T, g, ts, codes, scales, sf, status, clear_status, pdl, st, opt, sm_count);
+  return launch_stream<128>(X, M, K, T, g, ts, codes, scales, sf, status, clear_status, pdl, st, opt, sm_count);
 }
 
 }  // namespace wush
