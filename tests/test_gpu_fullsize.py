@@ -16,26 +16,29 @@ pytestmark = pytest.mark.gpu
 G = Q.GROUP
 
 
-def _check_layer(cfg, fmt, M, W_bits, Xc_bits, seed=0, rows=64, check_codes=True):
+def _check_layer(cfg, fmt, M, W_bits, Xc_bits, seed=0, rows=64, check_codes=True, dynamic=False):
     g = G[fmt]
     X_bits = synth.activations(cfg, M=M)
     L = P.PreparedLayer(W_bits, Xc_bits, fmt)
     K, N = cfg.K, W_bits.shape[0]
     X, W = dev_bf16(X_bits), dev_bf16(W_bits)
     wq, ws, tsw = wush.quantize_weight(W, dev(L.T_xvsh32), fmt, sf=wush.SF_TILED)
-    tsx = dev(np.full(4, L.ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
-    Y, wsp = wush.linear(X, dev_bf16(L.T_bits), wq, ws, fmt, tsx, tsw)
+    tsx = dev(np.full(4, L.ts_x, dtype=np.float32)) if (fmt == "nvfp4" and not dynamic) else None
+    Y, wsp = wush.linear(X, dev_bf16(L.T_bits), wq, ws, fmt, tsx, tsw)      # NVFP4 without tsx: per-batch scale
     torch.cuda.synchronize()
     assert wush.linear_status(wsp, M, K, g) == 0
+    ts_x = L.dynamic_ts_x(X_bits) if dynamic else L.ts_x
+    if dynamic:
+        assert abs(wush.linear_dynamic_scale(wsp, M, K, g)[0] - float(ts_x)) <= 2e-7 * float(ts_x)
     if check_codes:                                    # the activation codes wush_linear left in its workspace
         codes = wsp[: M * K // 2].view(M, K // 2).cpu().numpy()
         off = (M * K // 2 + 15) // 16 * 16
         sc = untile(wsp[off: off + wush.scale_bytes(M, K, g, wush.SF_TILED)].cpu().numpy(), M, K // g)
-        v32, _, _ = L.quantize_act(X_bits)
-        compare_quantized(codes, sc, v32, fmt, L.ts_x)
+        v32, _, _ = L.quantize_act(X_bits, ts_x)
+        compare_quantized(codes, sc, v32, fmt, ts_x)
     rng = np.random.default_rng(seed)
     pick = np.sort(rng.choice(M, size=min(rows, M), replace=False))
-    Yo = L.forward(X_bits, rows=pick)
+    Yo = L.forward(X_bits, rows=pick, dynamic=dynamic)
     assert rel_fro(Y[torch.from_numpy(pick).cuda()].cpu().numpy(), Yo) <= 1e-3
     return L
 
@@ -45,10 +48,15 @@ def test_config3_mxfp4_full():
     _check_layer(cfg, "mxfp4", cfg.M, synth.weights(cfg), synth.calibration(cfg))
 
 
-@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4"])
+@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4", "mxfp4_ceil"])
 def test_config4_full(fmt):
     cfg = synth.CONFIGS[4]
     _check_layer(cfg, fmt, cfg.M, synth.weights(cfg), synth.calibration(cfg))
+
+
+def test_config2_per_batch_tensor_scale_full():
+    cfg = synth.CONFIGS[2]
+    _check_layer(cfg, "nvfp4", cfg.M, synth.weights(cfg), synth.calibration(cfg), dynamic=True)
 
 
 @pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4"])
