@@ -79,14 +79,20 @@ __device__ __forceinline__ bool sq_elect() {
 // AMAX = true: the same tile walk and the same products, but instead of quantising, the AbsMax of everything
 // computed is folded into *ts_out (read as the uint32 bit pattern of a non-negative float, atomicMax): the
 // first pass of the per-batch NVFP4 tensor scale.  codes / scales are not touched.
-template <int G, bool AMAX = false, int ROWS = 128>
+// NSPLIT = 3: the weight side (Algorithm 2, last line).  Tsrc is then the fp32 T_xvsh; every entry is split
+// exactly into three bf16 terms (hi + mid + lo) when the fragments are loaded, and the three partial
+// products are accumulated smallest first.  Needs ROWS = 64 (three sets of fragments per super-block).
+template <int G, bool AMAX = false, int ROWS = 128, int NSPLIT = 1>
 __global__ void __launch_bounds__(SQ_THREADS, 1)
-tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
+tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restrict__ Tsrc, int64_t M, int64_t K,
                  const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
                  int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status, int clear_status,
                  const uint32_t* __restrict__ amax_in, float* __restrict__ ts_out, int mx_ceil) {
   constexpr int FMT = (G == 32) ? kFmtMX : kFmtNV;
+  static_assert(NSPLIT == 1 || (NSPLIT == 3 && ROWS == 64), "three-way split needs one super-block per warp");
   constexpr int SQ_ROWS = ROWS;
+  const __nv_bfloat16* T = reinterpret_cast<const __nv_bfloat16*>(Tsrc);      // NSPLIT = 1
+  const float* Tf = reinterpret_cast<const float*>(Tsrc);                     // NSPLIT = 3
   constexpr int NQ = ROWS / 64;                      // super-blocks per consumer warp
   constexpr int SLICES = ROWS / 16;                  // 16-row slices per tile
   constexpr int SQ_BOX_BYTES = ROWS * 128;           // one TMA box: ROWS rows x 64 channels
@@ -191,7 +197,8 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
     const int64_t KB = K / G;
     float seen = 0.0f;                         // AMAX: running maximum of this lane
 
-    uint4 tf[NQ][4];                          // B fragments of this warp's transforms, kept across items
+    uint4 tf[NSPLIT][NQ][4];                  // B fragments of this warp's transforms, kept across items
+                                              // (NSPLIT = 3: [0] = lo, [1] = mid, [2] = hi terms)
     int cur_panel = -1;
     int n = 0;
     int panel = item_begin / num_rb, rb = item_begin % num_rb;
@@ -227,18 +234,55 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
           for (int t = 0; t < 4; ++t) {
             const int r = 8 * nchunk + 2 * t + (gid & 1);     // transform row for column slot gid of tile t
             // B fragment of column slot gid: channels 2*tig, 2*tig+1 (+8) of k-step 0 in .x (.y), of k-step 1 in .z (.w)
-            uint4 w = make_uint4(0, 0, 0, 0);
-            if (wsb + q < nsb) {
-              if (G == 32) {
-                const uint32_t* row = reinterpret_cast<const uint32_t*>(T + ((int64_t)sb * 32 + r) * 32);
-                w = make_uint4(__ldg(row + tig), __ldg(row + 4 + tig), __ldg(row + 8 + tig), __ldg(row + 12 + tig));
-              } else if ((r >> 4) == (tig >> 1)) {
-                // permuted contraction index: the lane's 8 channels 8*tig.. belong to block tig >> 1 of the
-                // block-diagonal pair; off-diagonal pieces are zero
-                w = __ldg(reinterpret_cast<const uint4*>(T + (((int64_t)sb * 2 + (r >> 4)) * 16 + (r & 15)) * 16 + 8 * (tig & 1)));
+            if (NSPLIT == 1) {
+              uint4 w = make_uint4(0, 0, 0, 0);
+              if (wsb + q < nsb) {
+                if (G == 32) {
+                  const uint32_t* row = reinterpret_cast<const uint32_t*>(T + ((int64_t)sb * 32 + r) * 32);
+                  w = make_uint4(__ldg(row + tig), __ldg(row + 4 + tig), __ldg(row + 8 + tig), __ldg(row + 12 + tig));
+                } else if ((r >> 4) == (tig >> 1)) {
+                  // permuted contraction index: the lane's 8 channels 8*tig.. belong to block tig >> 1 of the
+                  // block-diagonal pair; off-diagonal pieces are zero
+                  w = __ldg(reinterpret_cast<const uint4*>(T + (((int64_t)sb * 2 + (r >> 4)) * 16 + (r & 15)) * 16 + 8 * (tig & 1)));
+                }
               }
+              tf[0][q][t] = w;
+            } else {
+              // the same eight entries as above, from the fp32 matrix, each split into hi + mid + lo
+              float f[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) f[i] = 0.f;
+              if (wsb + q < nsb) {
+                if (G == 32) {
+                  const float2* row = reinterpret_cast<const float2*>(Tf + ((int64_t)sb * 32 + r) * 32);
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) { const float2 v = __ldg(row + 4 * i + tig); f[2 * i] = v.x; f[2 * i + 1] = v.y; }
+                } else if ((r >> 4) == (tig >> 1)) {
+                  const float4* row = reinterpret_cast<const float4*>(Tf + (((int64_t)sb * 2 + (r >> 4)) * 16 + (r & 15)) * 16 + 8 * (tig & 1));
+                  const float4 v0 = __ldg(row), v1 = __ldg(row + 1);
+                  f[0] = v0.x; f[1] = v0.y; f[2] = v0.z; f[3] = v0.w; f[4] = v1.x; f[5] = v1.y; f[6] = v1.z; f[7] = v1.w;
+                }
+              }
+              uint32_t pk[3][4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                __nv_bfloat16 h[2][3];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                  const float x = f[2 * i + e];
+                  h[e][2] = __float2bfloat16_rn(x);
+                  const float r1 = x - __bfloat162float(h[e][2]);               // exact
+                  h[e][1] = __float2bfloat16_rn(r1);
+                  const float r2 = r1 - __bfloat162float(h[e][1]);              // exact
+                  h[e][0] = __float2bfloat16_rn(r2);
+                }
+#pragma unroll
+                for (int sp = 0; sp < 3; ++sp)
+                  pk[sp][i] = (uint32_t)__bfloat16_as_ushort(h[0][sp]) | ((uint32_t)__bfloat16_as_ushort(h[1][sp]) << 16);
+              }
+#pragma unroll
+              for (int sp = 0; sp < NSPLIT; ++sp) tf[sp][q][t] = make_uint4(pk[sp][0], pk[sp][1], pk[sp][2], pk[sp][3]);
             }
-            tf[q][t] = w;
           }
         }
         // output pointers of this panel at the current row block
@@ -303,8 +347,13 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* 
           float acc[4][4];
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
-            mma_bf16_16816_first(acc[t], af[q][0].x, af[q][0].y, af[q][0].z, af[q][0].w, tf[q][t].x, tf[q][t].y);
-            mma_bf16_16816(acc[t], af[q][1].x, af[q][1].y, af[q][1].z, af[q][1].w, tf[q][t].z, tf[q][t].w);
+            mma_bf16_16816_first(acc[t], af[q][0].x, af[q][0].y, af[q][0].z, af[q][0].w, tf[0][q][t].x, tf[0][q][t].y);
+            mma_bf16_16816(acc[t], af[q][1].x, af[q][1].y, af[q][1].z, af[q][1].w, tf[0][q][t].z, tf[0][q][t].w);
+#pragma unroll
+            for (int sp = 1; sp < NSPLIT; ++sp) {
+              mma_bf16_16816(acc[t], af[q][0].x, af[q][0].y, af[q][0].z, af[q][0].w, tf[sp][q][t].x, tf[sp][q][t].y);
+              mma_bf16_16816(acc[t], af[q][1].x, af[q][1].y, af[q][1].z, af[q][1].w, tf[sp][q][t].z, tf[sp][q][t].w);
+            }
           }
           float vA[8], vB[8];
 #pragma unroll
@@ -432,7 +481,7 @@ static SqEncodeFn sq_encode_fn() {
 }
 
 // One launch for a given tile height.  cudaErrorNotSupported: use the register-staged kernel instead.
-template <int ROWS>
+template <int ROWS, int NSPLIT = 1>
 static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                  uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl,
                                  cudaStream_t st, const QuantOpts& opt, int sm_count) {
@@ -449,9 +498,9 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
   static bool attr_done = false;
   cudaError_t e;
   if (!attr_done) {
-    if ((e = cudaFuncSetAttribute(tq_stream_kernel<32, false, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, false, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, true, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<32, false, ROWS, NSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, false, ROWS, NSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(tq_stream_kernel<16, true, ROWS, NSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
     attr_done = true;
   }
   const int num_rb = (int)((M + ROWS - 1) / ROWS);
@@ -460,7 +509,7 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
   if (items > 0x7fffffff || M > 0x7fffff00) return cudaErrorNotSupported;
   if ((M + ROWS) * (K / 2) >= ((int64_t)1 << 32)) return cudaErrorNotSupported;   // the kernel keeps 32-bit output offsets
   const int grid = (int)(items < sm_count ? items : sm_count);
-  const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
+  const void* Tb = T;
   const int cs = clear_status ? 1 : 0;
   const int n_items = (int)items;
   const uint32_t* amax_in = opt.amax_in;
@@ -468,15 +517,15 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
   const int mx_ceil = opt.mx_ceil ? 1 : 0;
   if (opt.amax_out != nullptr) {                 // AbsMax pass only (g = 16)
     if (g != 16) return cudaErrorNotSupported;
-    tq_stream_kernel<16, true, ROWS><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, nullptr, nullptr, nullptr, sf, num_rb, n_items,
+    tq_stream_kernel<16, true, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, nullptr, nullptr, nullptr, sf, num_rb, n_items,
                                                                         nullptr, 0, nullptr, reinterpret_cast<float*>(opt.amax_out), 0);
     return cudaGetLastError();
   }
   if (!pdl) {
     if (g == 32)
-      tq_stream_kernel<32, false, ROWS><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+      tq_stream_kernel<32, false, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
     else
-      tq_stream_kernel<16, false, ROWS><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+      tq_stream_kernel<16, false, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
     return cudaGetLastError();
   }
   // programmatic dependent launch: set-up overlaps the tail of the previous kernel of the stream
@@ -491,8 +540,32 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (g == 32)
-    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32, false, ROWS>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
-  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16, false, ROWS>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32, false, ROWS, NSPLIT>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16, false, ROWS, NSPLIT>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+}
+
+static cudaError_t stream_sm_count(int* out) {
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0;
+    cudaError_t e;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  }
+  *out = sm_count;
+  return cudaSuccess;
+}
+
+// Weight side through the same kernel: W[N,K] bf16, Tinv fp32 (three-way split), 64-row tiles.  opt carries
+// the AbsMax pass / tensor-scale pointers for NVFP4 exactly as on the activation side.
+cudaError_t run_quantize_weight_stream(const void* W, int64_t N, int64_t K, const float* Tinv, int g, uint8_t* codes,
+                                       uint8_t* scales, int sf, cudaStream_t st, const QuantOpts& opt) {
+  if (!sq_encode_fn()) return cudaErrorNotSupported;
+  if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;
+  int sm_count = 0;
+  const cudaError_t e = stream_sm_count(&sm_count);
+  if (e != cudaSuccess) return e;
+  return launch_stream<64, 3>(W, N, K, Tinv, g, nullptr, codes, scales, sf, nullptr, false, false, st, opt, sm_count);
 }
 
 // Returns cudaErrorNotSupported when the streaming kernel cannot take the problem (the caller
@@ -502,13 +575,9 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
                                     cudaStream_t st, const QuantOpts& opt) {
   if (!sq_encode_fn()) return cudaErrorNotSupported;
   if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
-  static int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    cudaError_t e;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  }
+  int sm_count = 0;
+  const cudaError_t e0 = stream_sm_count(&sm_count);
+  if (e0 != cudaSuccess) return e0;
   // 128-row tiles unless the problem is small: with fewer than SQ_SMALL of them per CTA the 64-row tiles'
   // finer items win (the first tile lands sooner and the CTAs finish closer together)
   const int64_t items128 = ((K / 32 + 3) / 4) * ((M + 127) / 128);
