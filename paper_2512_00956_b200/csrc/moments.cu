@@ -1,4 +1,5 @@
-// Per-block second-moment accumulation for calibration (Algorithm 2, RTN case, first line
+// Register-staged per-block second-moment accumulation (the fall-back of moments_stream.cu) and the
+// host entry of the calibration call (Algorithm 2, RTN case, first line
 // of the loop):  S_c += sum_t x_{t,c}^T x_{t,c}  for every block c of g channels.
 //
 // This is a batched SYRK with a tiny output (g x g per block) and a long contraction over
@@ -92,18 +93,16 @@ __global__ void moments_reduce_kernel(const float* __restrict__ partials, int sp
   moments[i] += s;
 }
 
-int moments_splits(int64_t B, int64_t K) {
-  const int64_t groups = (K / 32 + kMomWarps - 1) / kMomWarps;
-  int64_t s = (148 * 3 + groups - 1) / groups;
-  const int64_t max_by_tokens = (B + 63) / 64;                 // at least 64 tokens per split
-  if (s > max_by_tokens) s = max_by_tokens;
-  if (s > 64) s = 64;
-  if (s < 1) s = 1;
-  return (int)s;
-}
+// Sets of partial sums a call needs room for: what the streaming kernel may write per panel (the register-staged
+// kernel below takes any number of token splits and is given the same).
+int moments_splits(int64_t B, int64_t K) { return moments_stream_segments(B, K); }
 
 cudaError_t run_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* moments,
                               int64_t* count, float* partials, int splits, cudaStream_t st) {
+  // streaming kernel first (TMA-fed ring, ldmatrix.trans operands); it declines when the workspace holds fewer
+  // sets of partial sums than it may need, or without the tensor-map driver entry point
+  const cudaError_t es = run_calib_moments_stream(Xc, B, K, g, moments, count, partials, splits, st);
+  if (es != cudaErrorNotSupported) return es;
   const int64_t groups = (K / 32 + kMomWarps - 1) / kMomWarps;
   int tokens_per_split = (int)((B + splits - 1) / splits);
   tokens_per_split = (tokens_per_split + 15) / 16 * 16;

@@ -36,6 +36,10 @@ cudaError_t run_quantize_f32(const float* V, int64_t R, int64_t K, int g, const 
                              uint8_t* codes, uint8_t* scales, int sf, cudaStream_t st, bool mx_ceil = false);
 
 int moments_splits(int64_t B, int64_t K);
+int moments_stream_segments(int64_t B, int64_t K);
+// streaming moments (partial sums + segment-aware reduction); cudaErrorNotSupported = use the other kernels
+cudaError_t run_calib_moments_stream(const void* Xc, int64_t B, int64_t K, int g, float* moments, int64_t* count,
+                                     float* partials, int slots, cudaStream_t st);
 cudaError_t run_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* moments,
                               int64_t* count, float* partials, int splits, cudaStream_t st);
 
