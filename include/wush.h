@@ -34,6 +34,8 @@
  *     Argument errors are found on the host before anything is launched, and then
  *     no output is touched.
  *   - base pointers must be 16-byte aligned; K must be a multiple of 64.
+ *   - calls act on the CURRENT device of the calling thread; one-time launch set-up is
+ *     remembered per device, so a process may use several devices (device ordinals 0..63).
  */
 #ifndef WUSH_H_
 #define WUSH_H_

@@ -427,21 +427,23 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
   cfg.attrs = attr;
   cfg.numAttrs = after_quantizer ? 1 : 0;          // programmatic dependent of the quantiser inside wush_linear
   const int mi = (int)M, ni = (int)N, ki = (int)K, a_bytes = a_rows * BKB;
+  const int slot = device_slot();
+  if (slot < 0) return cudaErrorInvalidDevice;
   if (fmt == kFmtMX) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[kDeviceSlots] = {};
+    if (!attr_done[slot]) {
       e = cudaFuncSetAttribute(gemm_fp4_kernel<kFmtMX>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(kFmtMX));
       if (e != cudaSuccess) return e;
-      attr_done = true;
+      attr_done[slot] = true;
     }
     cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtMX);
     return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtMX>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes, cs);
   }
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kDeviceSlots] = {};
+  if (!attr_done[slot]) {
     e = cudaFuncSetAttribute(gemm_fp4_kernel<kFmtNV>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(kFmtNV));
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[slot] = true;
   }
   cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtNV);
   return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtNV>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes, cs);

@@ -491,7 +491,10 @@ template <int FMT>
 static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& sa, const CUtensorMap& sb,
                                int M, int N, int K, const float* tsx, const float* tsw, const CUtensorMap& y, int out_bf16,
                                int32_t* status, bool clear_status, bool pdl, cudaStream_t st) {
-  static int clusters = 0;
+  static int clusters_of[kDeviceSlots] = {};       // resident clusters of this kernel, per device
+  const int slot = device_slot();
+  if (slot < 0) return cudaErrorInvalidDevice;
+  int& clusters = clusters_of[slot];
   const int cs = clear_status ? 1 : 0;
   cudaError_t e;
   if (clusters == 0) {

@@ -321,16 +321,17 @@ cudaError_t run_moments_partial_stream(const void* Xc, int64_t B, int64_t K, int
   const int64_t num_rb = (B + MS_ROWS - 1) / MS_ROWS;
   const int64_t items = panels * num_rb;
   if (items > 0x7fffffff || B > 0x7fffff00) return cudaErrorNotSupported;
-  static int sm_count = 0;
-  static bool attr_done = false;
+  static int sm_count_of[kDeviceSlots] = {};
+  const int slot = device_slot();
+  if (slot < 0) return cudaErrorInvalidDevice;
+  int& sm_count = sm_count_of[slot];
   cudaError_t e;
-  if (!attr_done) {
-    int dev = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if (sm_count == 0) {
+    int dev = slot, sms = 0;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(moments_stream_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MS_SMEM)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(moments_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, MS_SMEM)) != cudaSuccess) return e;
-    attr_done = true;
+    sm_count = sms;
   }
   int64_t grid = (int64_t)sm_count * MS_CTAS_PER_SM < MS_DESIGN_SMS ? (int64_t)sm_count * MS_CTAS_PER_SM : MS_DESIGN_SMS;
   if (items < grid) grid = items;

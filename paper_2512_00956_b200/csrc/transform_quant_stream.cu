@@ -495,7 +495,10 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorNotSupported;
-  static bool attr_done = false;
+  static bool attr_done_of[kDeviceSlots] = {};
+  const int slot = device_slot();
+  if (slot < 0) return cudaErrorInvalidDevice;
+  bool& attr_done = attr_done_of[slot];
   cudaError_t e;
   if (!attr_done) {
     if ((e = cudaFuncSetAttribute(tq_stream_kernel<32, false, ROWS, NSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SQ_SMEM)) != cudaSuccess) return e;
@@ -545,14 +548,16 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
 }
 
 static cudaError_t stream_sm_count(int* out) {
-  static int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    cudaError_t e;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  static int sm_count_of[kDeviceSlots] = {};
+  const int slot = device_slot();
+  if (slot < 0) return cudaErrorInvalidDevice;
+  if (sm_count_of[slot] == 0) {
+    int sms = 0;
+    const cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, slot);
+    if (e != cudaSuccess) return e;
+    sm_count_of[slot] = sms;
   }
-  *out = sm_count;
+  *out = sm_count_of[slot];
   return cudaSuccess;
 }
 

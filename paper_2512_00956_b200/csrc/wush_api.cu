@@ -37,14 +37,15 @@ inline wush::QuantOpts opts_of(int fmt) {
 }
 
 bool device_is_sm100() {
-  static int cached = -1;
-  if (cached < 0) {
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
-    cached = (major == 10) ? 1 : 0;
+  static signed char cached[wush::kDeviceSlots] = {};   // 0 unknown, 1 yes, -1 no; per device
+  const int slot = wush::device_slot();
+  if (slot < 0) return false;
+  if (cached[slot] == 0) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, slot) != cudaSuccess) return false;
+    cached[slot] = (major == 10) ? 1 : -1;
   }
-  return cached == 1;
+  return cached[slot] == 1;
 }
 
 }  // namespace

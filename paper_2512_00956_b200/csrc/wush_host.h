@@ -6,6 +6,15 @@
 
 namespace wush {
 
+// One-time launch set-up (function attributes, SM count, cluster occupancy) is remembered per device: the
+// caches below are arrays indexed by the current device.  -1: no usable current device.
+constexpr int kDeviceSlots = 64;
+inline int device_slot() {
+  int d = 0;
+  if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kDeviceSlots) return -1;
+  return d;
+}
+
 // Optional rules of the activation quantiser.  mx_ceil: MXFP4 exponent by the ceil rule.  amax_in / ts_out
 // (NVFP4): take the tensor scale from *amax_in (bit pattern of the AbsMax found by run_act_amax) instead of
 // `ts`, and write the scale used to *ts_out.
