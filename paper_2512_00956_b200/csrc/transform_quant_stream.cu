@@ -196,6 +196,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restric
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
     float seen = 0.0f;                         // AMAX: running maximum of this lane
+    const NvScaleFast nvf = nv_scale_fast(ts);                 // NVFP4: reciprocal of the tensor scale for the branch-free divisions
 
     uint4 tf[NSPLIT][NQ][4];                  // B fragments of this warp's transforms, kept across items
                                               // (NSPLIT = 3: [0] = lo, [1] = mid, [2] = hi terms)
@@ -382,7 +383,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restric
             // four distinct scales per quad (row A/B x block 0/1): lane tig computes the one of
             // (row tig>>1, its own block) and fetches the other row's from lane tig^2
             const bool mine_is_b = (tig >> 1) != 0;
-            const uint32_t sm = nv_scale_byte(mine_is_b ? aB : aA, ts);
+            const uint32_t sm = nv_scale_byte(mine_is_b ? aB : aA, nvf);
             const uint32_t so = __shfl_xor_sync(0xffffffffu, sm, 2);
             sA[q] = mine_is_b ? so : sm; mA = nv_mult[sA[q]];
             sB[q] = mine_is_b ? sm : so; mB = nv_mult[sB[q]];

@@ -110,6 +110,39 @@ __device__ __forceinline__ uint32_t nv_scale_byte(float amax, float ts) {
   const float r = __fdiv_rn(__fdiv_rn(amax, 6.0f), ts);
   return static_cast<uint32_t>(__nv_cvt_float_to_fp8(r, __NV_SATFINITE, __NV_E4M3));
 }
+
+// x / b, correctly rounded, without the branchy IEEE division sequence: y = RN(1 / b) is given, one FMA
+// step makes the quotient faithful, a second one rounds it correctly (Markstein's division).  Valid while no
+// intermediate leaves the normal range; the callers below guard that.  wush_check_division compares it with
+// __fdiv_rn over all x of the guarded range for any divisors it is given.
+__device__ __forceinline__ float div_rn_fma(float x, float b, float y) {
+  float q = __fmul_rn(x, y);
+  float r = __fmaf_rn(-b, q, x);
+  q = __fmaf_rn(r, y, q);
+  r = __fmaf_rn(-b, q, x);
+  return __fmaf_rn(r, y, q);
+}
+constexpr float kRcp6 = 0.16666667163372040f;        // RN(1/6) = 0x3E2AAAAB
+// Per-kernel constants of the fast scale path: rts = RN(1 / ts), usable while ts lies in [2^-40, 2^40]
+struct NvScaleFast {
+  float ts, rts;
+  bool ts_ok;
+};
+__device__ __forceinline__ NvScaleFast nv_scale_fast(float t) {
+  NvScaleFast f;
+  f.ts = t;
+  f.rts = __frcp_rn(t);
+  f.ts_ok = (t >= 0x1p-40f && t <= 0x1p40f);
+  return f;
+}
+// The same byte as nv_scale_byte(amax, f.ts): blocks with amax in [2^-50, 2^50] take the FMA divisions (both
+// intermediates then stay far inside the normal range), everything else - zero blocks included - the IEEE ones.
+__device__ __forceinline__ uint32_t nv_scale_byte(float amax, const NvScaleFast& f) {
+  float r;
+  if (f.ts_ok && amax >= 0x1p-50f && amax <= 0x1p50f) r = div_rn_fma(div_rn_fma(amax, 6.0f, kRcp6), f.ts, f.rts);
+  else r = __fdiv_rn(__fdiv_rn(amax, 6.0f), f.ts);
+  return static_cast<uint32_t>(__nv_cvt_float_to_fp8(r, __NV_SATFINITE, __NV_E4M3));
+}
 __device__ __forceinline__ float nv_mult_of_byte(uint32_t byte, float ts) {
   const float d = __fmul_rn(e4m3_to_float(byte), ts);
   return (d == 0.0f) ? 0.0f : __frcp_rn(d);
