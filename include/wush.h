@@ -216,6 +216,13 @@ int wush_calib_moments_static(const void* Xc, int64_t B, int64_t K, int g, float
 int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, int g,
                       const float* tensor_scale, uint8_t* codes, uint8_t* scales,
                       wush_sf_layout_t sf, void* stream);
+/* The NVFP4 scale byte needs (AbsMax / 6) / tensor_scale with both divisions correctly rounded.  Inside
+ * AbsMax in [2^-50, 2^50] and tensor_scale in [2^-40, 2^40] the kernels evaluate them without the IEEE
+ * division sequence (reciprocal of the divisor, two fused multiply-add corrections); outside they use the
+ * IEEE division.  This call checks the equivalence on the device: for each of the n divisors b (fp32, device
+ * array, normal, in [2^-40, 2^40]) it compares the two for EVERY fp32 x in [2^-60, 2^60] and stores the number
+ * of x that differ in mismatches[i] (uint64, device array; expected: all zero).  About 1 ms per divisor. */
+int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void* stream);
 /* The block transform alone: V[M,K] fp32 = X_blk * T_c^T, same arithmetic as
  * wush_quantize_act uses before quantising. */
 int wush_transform_act_f32(const void* X, int64_t M, int64_t K, const void* T, int g,

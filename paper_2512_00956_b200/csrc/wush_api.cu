@@ -244,6 +244,14 @@ int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, i
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
+int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void* stream) {
+  if (n < 0 || n > 65535) return WUSH_ERR_SHAPE;
+  if (!divisors || !mismatches) return WUSH_ERR_NULL;
+  if (n == 0) return WUSH_OK;
+  cudaError_t e = wush::run_check_division(divisors, n, reinterpret_cast<unsigned long long*>(mismatches), (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
 int wush_transform_act_f32(const void* X, int64_t M, int64_t K, const void* T, int g, float* V, void* stream) {
   if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
   int rc = check_shape(M, K, g);

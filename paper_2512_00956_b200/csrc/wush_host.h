@@ -44,6 +44,8 @@ cudaError_t run_quantize_weight(const void* W, int64_t N, int64_t K, const float
 cudaError_t run_quantize_f32(const float* V, int64_t R, int64_t K, int g, const float* ts,
                              uint8_t* codes, uint8_t* scales, int sf, cudaStream_t st, bool mx_ceil = false);
 
+cudaError_t run_check_division(const float* divisors, int n, unsigned long long* mismatches, cudaStream_t st);
+
 int moments_splits(int64_t B, int64_t K);
 int moments_stream_segments(int64_t B, int64_t K);
 // streaming moments (partial sums + segment-aware reduction); cudaErrorNotSupported = use the other kernels

@@ -25,7 +25,7 @@ EXPORTS = [
     "wush_quantize_weight", "wush_quantize_weight_workspace_bytes", "wush_gemm_fp4", "wush_linear",
     "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
-    "wush_build_transforms", "wush_quantize_act_dynamic",
+    "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -66,6 +66,7 @@ def lib():
         L.wush_calib_moments_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]
         L.wush_calib_moments_static.restype = i32
         L.wush_quantize_f32.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, i32, vp]
+        L.wush_check_division.argtypes = [vp, i32, vp, vp]
         L.wush_transform_act_f32.argtypes = [vp, i64, i64, vp, i32, vp, vp]
         L.wush_transform_weight_f32.argtypes = [vp, i64, i64, vp, i32, vp, vp]
         for name in ("wush_quantize_act", "wush_quantize_weight", "wush_gemm_fp4", "wush_linear",
@@ -255,6 +256,14 @@ def quantize_f32(V, fmt, tensor_scale=None, sf=SF_LINEAR):
     codes, scales = _alloc_q(R, K, g, sf, V.device)
     check(lib().wush_quantize_f32(_ptr(V), R, K, f, g, _ptr(tensor_scale), _ptr(codes), _ptr(scales), sf, _stream()))
     return codes, scales
+
+
+def check_division(divisors):
+    """Mismatch counts (int64 tensor) of the branch-free division against the IEEE one, per divisor, over all x."""
+    _dev(divisors)
+    out = torch.zeros(divisors.numel(), dtype=torch.int64, device=divisors.device)
+    check(lib().wush_check_division(_ptr(divisors), divisors.numel(), _ptr(out), _stream()))
+    return out
 
 
 def transform_act_f32(X, T, g):

@@ -122,3 +122,26 @@ def test_dynamic_scale_all_zero_batch():
     torch.cuda.synchronize()
     assert float(ts[0].item()) == 1.0 and float(ts[1].item()) == 0.0
     assert int(codes.max().item()) == 0 and int(scales.max().item()) == 0
+
+
+# ------------------------------------------------------------------ the NVFP4 scale path's division
+def test_branch_free_division_equals_ieee_division_for_every_x():
+    """The scale byte must come from correctly rounded divisions.  The kernels' branch-free form is compared
+    on the device with the IEEE division for every fp32 x in [2^-60, 2^60] and for: 6, the tensor scales of
+    the synthetic layers, significands of all ones / one ulp above a power of two, and seeded random divisors
+    across the guarded exponent range."""
+    rng = np.random.default_rng(3)
+    divs = [6.0, 1.0, 0.0371, 2688.0]
+    for idx in (2, 4, 5):
+        d = synth.layer_inputs(synth.CONFIGS[idx], M=64, N=64)
+        L = P.PreparedLayer(d["W"], d["Xc"], "nvfp4")
+        divs += [float(L.ts_x), float(L.ts_w), float(L.dynamic_ts_x(d["X"]))]
+    bits = []
+    for e in (-40, -17, -1, 0, 1, 23, 40):
+        for m in (0x7FFFFF, 0x7FFFFE, 0x000001, 0x400000, 0x3FFFFF, 0x2AAAAB):
+            bits.append(((127 + e) << 23) | m)
+    bits += [int(((127 + int(rng.integers(-40, 41))) << 23) | int(rng.integers(0, 1 << 23))) for _ in range(64)]
+    divs = np.concatenate([np.array(divs, dtype=np.float32), np.array(bits, dtype=np.uint32).view(np.float32)])
+    bad = wush.check_division(dev(divs))
+    torch.cuda.synchronize()
+    assert int(bad.abs().max().item()) == 0, [(float(divs[i]), int(b)) for i, b in enumerate(bad.cpu().tolist()) if b]
