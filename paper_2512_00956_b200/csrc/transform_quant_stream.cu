@@ -63,6 +63,11 @@ __device__ __forceinline__ uint4 sq_lds128(uint32_t addr) {          // 128-bit 
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
+__device__ __forceinline__ float sq_lds_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
 // four 8x8 matrices of 16-bit elements, one row address per lane: the result is the A operand of m16n8k16
 __device__ __forceinline__ uint4 sq_ldmatrix_x4(uint32_t addr) {
   uint4 v;
@@ -196,6 +201,7 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restric
     const int nchunk = (((gid >> 1) & 1) << 1) | (gid >> 2);  // c(gid/2): chunk of the column slot this lane feeds
     const int64_t KB = K / G;
     float seen = 0.0f;                         // AMAX: running maximum of this lane
+    const uint32_t nv_mult_u32 = sq_smem_u32(nv_mult);
     const NvScaleFast nvf = nv_scale_fast(ts);                 // NVFP4: reciprocal of the tensor scale for the branch-free divisions
 
     uint4 tf[NSPLIT][NQ][4];                  // B fragments of this warp's transforms, kept across items
@@ -385,8 +391,8 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restric
             const bool mine_is_b = (tig >> 1) != 0;
             const uint32_t sm = nv_scale_byte(mine_is_b ? aB : aA, nvf);
             const uint32_t so = __shfl_xor_sync(0xffffffffu, sm, 2);
-            sA[q] = mine_is_b ? so : sm; mA = nv_mult[sA[q]];
-            sB[q] = mine_is_b ? sm : so; mB = nv_mult[sB[q]];
+            sA[q] = mine_is_b ? so : sm; mA = sq_lds_f32(nv_mult_u32 + 4 * sA[q]);
+            sB[q] = mine_is_b ? sm : so; mB = sq_lds_f32(nv_mult_u32 + 4 * sB[q]);
           }
           const uint64_t mA2 = pair_of(mA), mB2 = pair_of(mB);       // {m, m} built once per row
 #pragma unroll
