@@ -36,6 +36,9 @@
  *   - base pointers must be 16-byte aligned; K must be a multiple of 64.
  *   - calls act on the CURRENT device of the calling thread; one-time launch set-up is
  *     remembered per device, so a process may use several devices (device ordinals 0..63).
+ *   - entry points may be called from several host threads at once (the remembered set-up is
+ *     written idempotently, the error text is per thread); calls that share an output buffer,
+ *     a workspace or the built-in scratch of wush_calib_moments_static must be ordered by the caller.
  */
 #ifndef WUSH_H_
 #define WUSH_H_
