@@ -1,7 +1,8 @@
 """Parity at the benchmark's full sizes (configs 3-5), in the launch configuration bench.py uses
 (`wush_linear`, TILED scales, persistent kernels).  Activations are checked in full (codes and
-scale bytes, guard-band rule); Y is checked on sampled token rows, and for the 28672-wide layer
-also on sampled output channels, because the fp64 oracle cannot afford the full product."""
+scale bytes, guard-band rule; at M = 16384 on 256 sampled token rows); Y is checked on sampled
+token rows, and for the 28672-wide layer also on sampled output channels, because the fp64 oracle
+cannot afford the full product."""
 import numpy as np
 import pytest
 import torch
@@ -38,6 +39,13 @@ def _check_layer(cfg, fmt, M, W_bits, Xc_bits, seed=0, rows=64, check_codes=True
         compare_quantized(codes, sc, v32, fmt, ts_x)
     rng = np.random.default_rng(seed)
     pick = np.sort(rng.choice(M, size=min(rows, M), replace=False))
+    if not check_codes:                                # too many rows for the oracle: codes and scales of sampled rows
+        sel = np.sort(rng.choice(M, size=256, replace=False))
+        codes = wsp[: M * K // 2].view(M, K // 2)[torch.from_numpy(sel).cuda()].cpu().numpy()
+        off = (M * K // 2 + 15) // 16 * 16
+        sc = untile(wsp[off: off + wush.scale_bytes(M, K, g, wush.SF_TILED)].cpu().numpy(), M, K // g)[sel]
+        v32, _, _ = L.quantize_act(X_bits[sel], ts_x)
+        compare_quantized(codes, sc, v32, fmt, ts_x)
     Yo = L.forward(X_bits, rows=pick, dynamic=dynamic)
     assert rel_fro(Y[torch.from_numpy(pick).cuda()].cpu().numpy(), Yo) <= 1e-3
     return L
