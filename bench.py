@@ -417,6 +417,51 @@ def run_ours(args):
     D.shutdown()
 
 
+def run_quantiser_sweep(args):
+    """`--quantiser-sweep`: wush_quantize_act alone over seven activation shapes, both formats, on a GPU that
+    runs nothing else (0.3 s idle before every timed replay), one line of JSON per shape.  Random bf16 data
+    and transforms: the kernel's time does not depend on the values."""
+    import torch
+    from paper_2512_00956_b200 import wush
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    reps = 20
+    for M, K in ((2048, 4096), (1024, 8192), (4096, 4096), (4096, 8192), (4096, 14336), (8192, 8192), (16384, 8192)):
+        for fmt, g in (("mxfp4", 32), ("nvfp4", 16)):
+            nset = max(2, int(300e6 // (M * K * 2)) + 1)            # cold data: more than twice the L2 between reuses
+            Xs = [torch.randn(M, K, device=dev).to(torch.bfloat16) for _ in range(nset)]
+            T = (torch.randn(K // g, g, g, device=dev) / g ** 0.5).to(torch.bfloat16)
+            outs = [(torch.empty(M, K // 2, dtype=torch.uint8, device=dev),
+                     torch.zeros(wush.scale_bytes(M, K, g, wush.SF_TILED), dtype=torch.uint8, device=dev)) for _ in range(nset)]
+            ts = torch.tensor([0.01], device=dev) if fmt == "nvfp4" else None
+            side = torch.cuda.Stream(device=dev)
+            with torch.cuda.stream(side):
+                for i in range(3):
+                    wush.quantize_act(Xs[i % nset], T, fmt, ts, wush.SF_TILED, out=outs[i % nset])
+                side.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for i in range(reps):
+                        wush.quantize_act(Xs[i % nset], T, fmt, ts, wush.SF_TILED, out=outs[i % nset])
+                graph.replay()
+                side.synchronize()
+                times = []
+                for _ in range(5):
+                    time.sleep(0.3)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(side)
+                    graph.replay()
+                    b.record(side)
+                    side.synchronize()
+                    times.append(a.elapsed_time(b) / reps * 1e3)
+            us = statistics.median(times)
+            nbytes = 2.0 * M * K + M * K / 2.0 + M * K / g + 2.0 * K * g
+            print(json.dumps({"kernel": "tq_stream_kernel", "M": M, "K": K, "format": fmt, "us": round(us, 2),
+                              "us_min": round(min(times), 2), "GB/s": round(nbytes / us / 1e3),
+                              "items_per_sm": round((M / 128) * (K / 128) / 148, 1)}), flush=True)
+            del Xs, outs, graph
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -433,7 +478,12 @@ def main():
                     help="activation-side transform: per-block WUSH (default), one shared Hadamard, or none")
     ap.add_argument("--ref-rows", type=int, default=1024, help="token rows in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quantiser-sweep", action="store_true",
+                    help="time wush_quantize_act alone over seven shapes (one JSON line each) and exit")
     args = ap.parse_args()
+    if args.quantiser_sweep:
+        run_quantiser_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
