@@ -226,6 +226,12 @@ int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, i
  * array, normal, in [2^-40, 2^40]) it compares the two for EVERY fp32 x in [2^-60, 2^60] and stores the number
  * of x that differ in mismatches[i] (uint64, device array; expected: all zero).  About 1 ms per divisor. */
 int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void* stream);
+/* Test hook for the persistent GEMM (M > 128): use at most `clusters` two-CTA clusters in later calls on the
+ * calling thread's current device (0 = as many as fit, the default).  With few clusters even a small problem
+ * gives every cluster several tiles in a row, which is how the tests reach the hand-over between tiles
+ * (accumulator drained while the next tile's loads run) without a full-size input.  Results never depend
+ * on it.  Returns the previous value. */
+int wush_debug_gemm_clusters(int clusters);
 /* The block transform alone: V[M,K] fp32 = X_blk * T_c^T, same arithmetic as
  * wush_quantize_act uses before quantising. */
 int wush_transform_act_f32(const void* X, int64_t M, int64_t K, const void* T, int g,

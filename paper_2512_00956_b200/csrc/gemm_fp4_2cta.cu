@@ -487,6 +487,15 @@ static bool map_output(CUtensorMap* map, void* Y, int64_t M, int64_t N, int out_
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+static int g_cluster_limit[kDeviceSlots] = {};
+int gemm_2cta_cluster_limit(int clusters) {
+  const int slot = device_slot();
+  if (slot < 0) return 0;
+  const int old = g_cluster_limit[slot];
+  g_cluster_limit[slot] = clusters < 0 ? 0 : clusters;
+  return old;
+}
+
 template <int FMT>
 static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& sa, const CUtensorMap& sb,
                                int M, int N, int K, const float* tsx, const float* tsw, const CUtensorMap& y, int out_bf16,
@@ -517,7 +526,8 @@ static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const
     clusters = n < sms / 2 ? n : sms / 2;
   }
   const int tiles = ((M + g2::BM - 1) / g2::BM) * ((N + g2::BN - 1) / g2::BN);
-  const int nc = tiles < clusters ? tiles : clusters;
+  int nc = tiles < clusters ? tiles : clusters;
+  if (g_cluster_limit[slot] > 0 && g_cluster_limit[slot] < nc) nc = g_cluster_limit[slot];
   if (!pdl) {
     g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, y,
                                                                                      out_bf16, status, cs);

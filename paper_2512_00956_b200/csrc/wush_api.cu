@@ -244,6 +244,8 @@ int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, i
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
+int wush_debug_gemm_clusters(int clusters) { return wush::gemm_2cta_cluster_limit(clusters); }
+
 int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void* stream) {
   if (n < 0 || n > 65535) return WUSH_ERR_SHAPE;
   if (!divisors || !mismatches) return WUSH_ERR_NULL;

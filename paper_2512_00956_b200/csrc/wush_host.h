@@ -65,6 +65,7 @@ cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* m
                                  double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st);
 
 // two-CTA persistent variant (M > 128); cudaErrorNotSupported = use the single-CTA kernel
+int gemm_2cta_cluster_limit(int clusters);   // test hook: 0 = no limit; returns the previous value (per device)
 cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws, int64_t M,
                               int64_t N, int64_t K, int fmt, const float* tsx, const float* tsw, void* Y,
                               int out_bf16, int32_t* status, bool clear_status, bool pdl, cudaStream_t st);

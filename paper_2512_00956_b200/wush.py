@@ -25,7 +25,7 @@ EXPORTS = [
     "wush_quantize_weight", "wush_quantize_weight_workspace_bytes", "wush_gemm_fp4", "wush_linear",
     "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
-    "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division",
+    "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division", "wush_debug_gemm_clusters",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -64,6 +64,8 @@ def lib():
         L.wush_build_transforms.argtypes = [vp, i64, vp, i64, i64, i32, ctypes.c_float, vp, vp, vp, vp]
         L.wush_build_transforms.restype = i32
         L.wush_calib_moments_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]
+        L.wush_debug_gemm_clusters.argtypes = [i32]
+        L.wush_debug_gemm_clusters.restype = i32
         L.wush_calib_moments_static.restype = i32
         L.wush_quantize_f32.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, i32, vp]
         L.wush_check_division.argtypes = [vp, i32, vp, vp]
@@ -256,6 +258,11 @@ def quantize_f32(V, fmt, tensor_scale=None, sf=SF_LINEAR):
     codes, scales = _alloc_q(R, K, g, sf, V.device)
     check(lib().wush_quantize_f32(_ptr(V), R, K, f, g, _ptr(tensor_scale), _ptr(codes), _ptr(scales), sf, _stream()))
     return codes, scales
+
+
+def debug_gemm_clusters(clusters):
+    """Test hook: limit the persistent GEMM to `clusters` clusters (0 = no limit); returns the old value."""
+    return int(lib().wush_debug_gemm_clusters(int(clusters)))
 
 
 def check_division(divisors):
