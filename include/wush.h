@@ -58,7 +58,7 @@ typedef enum {
   WUSH_ERR_ALIGN = -4,     /* a base pointer is not 16-byte aligned */
   WUSH_ERR_WORKSPACE = -5, /* workspace missing or smaller than wush_*_workspace_bytes() */
   WUSH_ERR_CUDA = -6,      /* a CUDA call or launch failed; see wush_last_cuda_error() */
-  WUSH_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (reported by wush_gemm_status) */
+  WUSH_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (wush_decode_status of a kernel's status word) */
   WUSH_ERR_DEVICE = -8     /* the current device is not compute capability 10.x */
 } wush_status_t;
 
@@ -82,6 +82,15 @@ typedef enum { WUSH_SF_LINEAR = 0, WUSH_SF_TILED = 1 } wush_sf_layout_t;
 typedef enum { WUSH_OUT_F32 = 0, WUSH_OUT_BF16 = 1 } wush_out_t;
 
 const char* wush_status_string(int status);
+/* Every wait inside the kernels is bounded (one to two seconds).  When one runs out, the kernel records a
+ * diagnostic word in the int32 `status` buffer of the call (wush_gemm_fp4: its argument; wush_linear: the last
+ * 16 bytes of the workspace), lets its outstanding copies land, frees what it holds and returns; the outputs
+ * of that call are then undefined and the context stays usable.  The word is 0 when nothing expired, else
+ * (role << 16) | index: role 0x04 / 0x05 = producer / consumer of the quantiser (index = work item of the CTA),
+ * 0x11..0x15 = producer, scale-copy wait, accumulator hand-over, epilogue, operand wait of the GEMM for
+ * M > 128, 0x01..0x03 = producer, MMA issuer, epilogue of the GEMM for M <= 128.  The
+ * caller copies the word to the host after synchronising; this helper maps it to WUSH_OK or WUSH_ERR_TIMEOUT. */
+int wush_decode_status(int32_t word);
 /* Text of the last CUDA error this library saw on the calling thread ("" if none). */
 const char* wush_last_cuda_error(void);
 
@@ -232,6 +241,11 @@ int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void
  * (accumulator drained while the next tile's loads run) without a full-size input.  Results never depend
  * on it.  Returns the previous value. */
 int wush_debug_gemm_clusters(int clusters);
+/* Test hook for the error path: the next wush_linear call on the calling thread's current device leaves the
+ * tile of work item `item` of its quantiser kernel unrequested (one call only; -1 cancels).  The consumers'
+ * bounded wait for that tile (about a second) then expires, the status word is set, both kernels of the
+ * call still complete and the next call works as usual.  Nothing faults and nothing waits without a bound. */
+int wush_debug_drop_tile(int item);
 /* The block transform alone: V[M,K] fp32 = X_blk * T_c^T, same arithmetic as
  * wush_quantize_act uses before quantising. */
 int wush_transform_act_f32(const void* X, int64_t M, int64_t K, const void* T, int g,

@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(SQ_THREADS, 1)
 tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restrict__ Tsrc, int64_t M, int64_t K,
                  const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
                  int sf_layout, int num_rb, int num_items, int32_t* __restrict__ status, int clear_status,
-                 const uint32_t* __restrict__ amax_in, float* __restrict__ ts_out, int mx_ceil) {
+                 const uint32_t* __restrict__ amax_in, float* __restrict__ ts_out, int mx_ceil, int drop_item) {
   constexpr int FMT = (G == 32) ? kFmtMX : kFmtNV;
   static_assert(NSPLIT == 1 || (NSPLIT == 3 && ROWS == 64), "three-way split needs one super-block per warp");
   constexpr int SQ_ROWS = ROWS;
@@ -162,7 +162,9 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restric
         break;
       }
       const int nsb = min(4, total_sb - panel * 4);
-      if (sq_elect()) {
+      // drop_item (a test hook, -1 in production): this item's tile is never requested, so the consumers'
+      // bounded wait for it runs out and the kernel leaves through its error path
+      if (it != drop_item && sq_elect()) {
         const uint32_t bar = sq_smem_u32(&full_bar[s]);
         const int nbox = nsb >> 1;                       // 64-channel (128-byte) boxes; K % 64 == 0
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(nbox * SQ_BOX_BYTES) : "memory");
@@ -525,17 +527,18 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
   const uint32_t* amax_in = opt.amax_in;
   float* ts_out = opt.ts_out;
   const int mx_ceil = opt.mx_ceil ? 1 : 0;
+  const int drop = opt.drop_item;
   if (opt.amax_out != nullptr) {                 // AbsMax pass only (g = 16)
     if (g != 16) return cudaErrorNotSupported;
     tq_stream_kernel<16, true, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, nullptr, nullptr, nullptr, sf, num_rb, n_items,
-                                                                        nullptr, 0, nullptr, reinterpret_cast<float*>(opt.amax_out), 0);
+                                                                        nullptr, 0, nullptr, reinterpret_cast<float*>(opt.amax_out), 0, -1);
     return cudaGetLastError();
   }
   if (!pdl) {
     if (g == 32)
-      tq_stream_kernel<32, false, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+      tq_stream_kernel<32, false, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil, drop);
     else
-      tq_stream_kernel<16, false, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+      tq_stream_kernel<16, false, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil, drop);
     return cudaGetLastError();
   }
   // programmatic dependent launch: set-up overlaps the tail of the previous kernel of the stream
@@ -550,8 +553,8 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (g == 32)
-    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32, false, ROWS, NSPLIT>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
-  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16, false, ROWS, NSPLIT>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil);
+    return cudaLaunchKernelEx(&cfg, tq_stream_kernel<32, false, ROWS, NSPLIT>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil, drop);
+  return cudaLaunchKernelEx(&cfg, tq_stream_kernel<16, false, ROWS, NSPLIT>, map, Tb, M, K, ts, codes, scales, sf, num_rb, n_items, status, cs, amax_in, ts_out, mx_ceil, drop);
 }
 
 static cudaError_t stream_sm_count(int* out) {

@@ -36,6 +36,18 @@ inline wush::QuantOpts opts_of(int fmt) {
   return o;
 }
 
+// test hook (wush_debug_drop_tile): work item the next streaming-quantiser launch of wush_linear on this device
+// will not load; one shot
+int g_drop_item[wush::kDeviceSlots];
+bool g_drop_init = false;
+int take_drop_item() {
+  const int slot = wush::device_slot();
+  if (slot < 0 || !g_drop_init) return -1;
+  const int v = g_drop_item[slot];
+  g_drop_item[slot] = -1;
+  return v;
+}
+
 bool device_is_sm100() {
   static signed char cached[wush::kDeviceSlots] = {};   // 0 unknown, 1 yes, -1 no; per device
   const int slot = wush::device_slot();
@@ -183,6 +195,7 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_
   if (!device_is_sm100()) return WUSH_ERR_DEVICE;
   // one status word for both kernels: cleared by the quantiser kernel, set by whichever bounded wait expires
   wush::QuantOpts o = opts_of(fmt);
+  o.drop_item = take_drop_item();
   cudaError_t e;
   if (dynamic) {                                  // per-batch tensor scale: AbsMax pass first
     uint32_t* amax = reinterpret_cast<uint32_t*>(ts_dyn + 1);
@@ -245,6 +258,19 @@ int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, i
 }
 
 int wush_debug_gemm_clusters(int clusters) { return wush::gemm_2cta_cluster_limit(clusters); }
+
+int wush_debug_drop_tile(int item) {
+  const int slot = wush::device_slot();
+  if (slot < 0) return WUSH_ERR_CUDA;
+  if (!g_drop_init) {
+    for (int i = 0; i < wush::kDeviceSlots; ++i) g_drop_item[i] = -1;
+    g_drop_init = true;
+  }
+  g_drop_item[slot] = item < 0 ? -1 : item;
+  return WUSH_OK;
+}
+
+int wush_decode_status(int32_t word) { return word == 0 ? WUSH_OK : WUSH_ERR_TIMEOUT; }
 
 int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void* stream) {
   if (n < 0 || n > 65535) return WUSH_ERR_SHAPE;

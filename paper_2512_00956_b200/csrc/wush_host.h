@@ -23,6 +23,7 @@ struct QuantOpts {
   const uint32_t* amax_in = nullptr;
   float* ts_out = nullptr;
   uint32_t* amax_out = nullptr;   // run_quantize_act_stream only: AbsMax pass instead of quantising (g = 16)
+  int drop_item = -1;             // test hook: the producer never requests this work item (streaming kernel only)
 };
 // clear_status: the kernel zeroes *status itself (wush_linear); otherwise the word is left alone
 cudaError_t run_quantize_act(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,

@@ -26,6 +26,7 @@ EXPORTS = [
     "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
     "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division", "wush_debug_gemm_clusters",
+    "wush_debug_drop_tile", "wush_decode_status",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -66,6 +67,8 @@ def lib():
         L.wush_calib_moments_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]
         L.wush_debug_gemm_clusters.argtypes = [i32]
         L.wush_debug_gemm_clusters.restype = i32
+        L.wush_debug_drop_tile.argtypes = [i32]
+        L.wush_decode_status.argtypes = [i32]
         L.wush_calib_moments_static.restype = i32
         L.wush_quantize_f32.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, i32, vp]
         L.wush_check_division.argtypes = [vp, i32, vp, vp]
@@ -258,6 +261,16 @@ def quantize_f32(V, fmt, tensor_scale=None, sf=SF_LINEAR):
     codes, scales = _alloc_q(R, K, g, sf, V.device)
     check(lib().wush_quantize_f32(_ptr(V), R, K, f, g, _ptr(tensor_scale), _ptr(codes), _ptr(scales), sf, _stream()))
     return codes, scales
+
+
+def debug_drop_tile(item):
+    """Test hook: the next `linear` call does not load work item `item` of its quantiser (-1 cancels)."""
+    check(lib().wush_debug_drop_tile(int(item)))
+
+
+def decode_status(word):
+    """WUSH_OK (0) or WUSH_ERR_TIMEOUT for a status word read back from the device."""
+    return int(lib().wush_decode_status(int(word)))
 
 
 def debug_gemm_clusters(clusters):

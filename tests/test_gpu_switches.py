@@ -1,6 +1,7 @@
 """GPU parity of the two optional quantiser rules against the oracle, through the C ABI:
 the MXFP4 ceil rule ("mxfp4_ceil") and the per-batch NVFP4 activation tensor scale.
-Same tolerances as the main parity tests."""
+Same tolerances as the main parity tests.  Also here: the exhaustive check of the branch-free
+division and the error path of a bounded wait that runs out."""
 import numpy as np
 import pytest
 import torch
@@ -145,3 +146,26 @@ def test_branch_free_division_equals_ieee_division_for_every_x():
     bad = wush.check_division(dev(divs))
     torch.cuda.synchronize()
     assert int(bad.abs().max().item()) == 0, [(float(divs[i]), int(b)) for i, b in enumerate(bad.cpu().tolist()) if b]
+
+
+# ------------------------------------------------------------------ error path: a bounded wait that runs out
+def test_expired_wait_is_reported_and_the_next_call_works():
+    """The test hook leaves one tile of the quantiser unrequested: the consumers' bounded wait for it
+    (about a second) expires, the status word names the quantiser's consumer role, both kernels of the call
+    still complete, nothing faults, and the same call repeated without the hook gives the oracle's result."""
+    fmt, M, N, K = "mxfp4", 300, 520, 1024
+    d, L = _layer(1, fmt, M=M, N=N, K=K, B=256)
+    X, W = dev_bf16(d["X"]), dev_bf16(d["W"])
+    wq, ws, tsw = wush.quantize_weight(W, dev(L.T_xvsh32), fmt, sf=wush.SF_TILED)
+    T = dev_bf16(L.T_bits)
+    wush.debug_drop_tile(0)
+    Y, wsp = wush.linear(X, T, wq, ws, fmt, None, tsw)
+    torch.cuda.synchronize()
+    word = wush.linear_status(wsp, M, K, 32)
+    assert word != 0 and (word >> 16) in (0x04, 0x05), hex(word)
+    assert wush.decode_status(word) == wush.lib().wush_decode_status(1) != 0      # WUSH_ERR_TIMEOUT
+    assert wush.decode_status(0) == 0
+    Y, wsp = wush.linear(X, T, wq, ws, fmt, None, tsw)                           # the hook was for one call
+    torch.cuda.synchronize()
+    assert wush.linear_status(wsp, M, K, 32) == 0
+    assert rel_fro(Y.cpu().numpy(), L.forward(d["X"])) <= 1e-3
