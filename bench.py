@@ -474,8 +474,9 @@ def main():
                     help="NVFP4: activation tensor scale from each batch (one more kernel per step) instead of calibration")
     ap.add_argument("--m", type=int, default=None, help="override the token count (config 5 sweep)")
     ap.add_argument("--out", default="bf16", choices=["bf16", "f32"])
-    ap.add_argument("--transform", default="wush", choices=["wush", "hadamard", "identity"],
-                    help="activation-side transform: per-block WUSH (default), one shared Hadamard, or none")
+    ap.add_argument("--transform", default="wush", choices=["wush", "wus", "hadamard", "identity"],
+                    help="activation-side transform: per-block WUSH (default), WUSH without its Hadamard factor, "
+                         "one shared Hadamard, or none")
     ap.add_argument("--ref-rows", type=int, default=1024, help="token rows in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quantiser-sweep", action="store_true",

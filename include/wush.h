@@ -195,6 +195,17 @@ size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g);
 int wush_build_transforms(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x,
                           int64_t K, int g, float lambda, void* T, float* Tinv, int32_t* info,
                           void* stream);
+/* The same with a choice of transform: WUSH_KIND_WUSH (the call above) or WUSH_KIND_WUS, the ablation of
+ * Sec. 6 / Table 1 "WUSH without Hadamard", T = S^-1/2 U^T W'^T.  Errors as above; FORMAT for another kind. */
+typedef enum { WUSH_KIND_WUSH = 0, WUSH_KIND_WUS = 1 } wush_transform_kind_t;
+int wush_build_transforms_kind(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x,
+                               int64_t K, int g, float lambda, wush_transform_kind_t kind, void* T,
+                               float* Tinv, int32_t* info, void* stream);
+/* Weight-side partners of given activation-side transforms (Eq. 6): Tinv[c] = (T[c])^-T for every block,
+ * fp64 Gauss-Jordan with partial pivoting, result in fp32.  T bf16 [K/g][g][g] (any transforms: a shared
+ * Hadamard matrix, the identity, user-supplied ones), Tinv fp32 [K/g][g][g], info optional int32[K/g]
+ * (0 = ok, 3 = singular).  Errors: NULL / SHAPE / FORMAT / ALIGN / CUDA. */
+int wush_invert_transforms(const void* T, int64_t K, int g, float* Tinv, int32_t* info, void* stream);
 
 /* wush_calib_moments without a workspace argument.  (No counterpart in the paper: this is
  * a packaging variant of the call above, added for hosts where this library must not and

@@ -45,11 +45,57 @@ __device__ void cholesky_lower(double* A, int* fail) {       // in place; upper 
   __syncthreads();
 }
 
+// Gauss-Jordan with partial pivoting on the D x D matrix Tm (destroyed); Rm becomes the inverse, fac holds D
+// scratch values; the TRANSPOSE of the inverse is written to out (fp32).  *fail = 3 if a pivot is zero.
+template <int D>
+__device__ void inverse_transpose(double* Tm, double* Rm, double* fac_buf, int* perm, int* fail_ptr, float* out) {
+  const int tid = threadIdx.x;
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) Rm[idx] = ((idx / D) == (idx % D)) ? 1.0 : 0.0;
+  __syncthreads();
+  for (int col = 0; col < D; ++col) {
+    if (tid == 0) {
+      int pr = col; double pv = fabs(Tm[col * D + col]);
+      for (int r = col + 1; r < D; ++r) if (fabs(Tm[r * D + col]) > pv) { pv = fabs(Tm[r * D + col]); pr = r; }
+      perm[0] = pr;
+      if (!(pv > 0.0)) *fail_ptr = 3;
+    }
+    __syncthreads();
+    const int pr = perm[0];
+    if (pr != col) {
+      for (int k = tid; k < D; k += BT_THREADS) {
+        double t = Tm[col * D + k]; Tm[col * D + k] = Tm[pr * D + k]; Tm[pr * D + k] = t;
+        t = Rm[col * D + k]; Rm[col * D + k] = Rm[pr * D + k]; Rm[pr * D + k] = t;
+      }
+    }
+    __syncthreads();
+    const double piv = Tm[col * D + col];
+    __syncthreads();
+    for (int k = tid; k < D; k += BT_THREADS) { Tm[col * D + k] /= piv; Rm[col * D + k] /= piv; }
+    __syncthreads();
+    // eliminate column `col` from every other row; factors are read before any row is modified
+    {
+      double* fac = fac_buf;
+      for (int r = tid; r < D; r += BT_THREADS) fac[r] = (r == col) ? 0.0 : Tm[r * D + col];
+      __syncthreads();
+      for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+        const int r = idx / D, k = idx % D;
+        const double f = fac[r];
+        if (f != 0.0) { Tm[idx] -= f * Tm[col * D + k]; Rm[idx] -= f * Rm[col * D + k]; }
+      }
+    }
+    __syncthreads();
+  }
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
+    const int j = idx / D, k = idx % D;
+    out[idx] = (float)Rm[k * D + j];      // transpose of the inverse
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(BT_THREADS)
 build_transforms_kernel(const float* __restrict__ mom_w, double inv_nw, const float* __restrict__ mom_x, double inv_nx,
                         double lambda, __nv_bfloat16* __restrict__ T_out, float* __restrict__ Tinv_out,
-                        int32_t* __restrict__ info) {
+                        int32_t* __restrict__ info, int with_hadamard) {
   extern __shared__ double sm[];
   double* Wp = sm;                 // M_W -> W'
   double* Xp = Wp + D * D;         // M_X -> X'
@@ -177,58 +223,53 @@ build_transforms_kernel(const float* __restrict__ mom_w, double inv_nw, const fl
   for (int idx = tid; idx < D * D; idx += BT_THREADS) {
     const int a = idx / D, k = idx % D;
     double s = 0.0;
-    for (int i = 0; i < D; ++i) s += ((__popc(a & i) & 1) ? -Rm[i * D + k] : Rm[i * D + k]);
-    const __nv_bfloat16 tb = __double2bfloat16(s * hnorm);
+    if (with_hadamard) {
+      for (int i = 0; i < D; ++i) s += ((__popc(a & i) & 1) ? -Rm[i * D + k] : Rm[i * D + k]);
+      s *= hnorm;
+    } else {
+      s = Rm[idx];                                   // "WUS": the same transform without the Hadamard factor
+    }
+    const __nv_bfloat16 tb = __double2bfloat16(s);
     T_out[(size_t)c * D * D + idx] = tb;
     Tm[idx] = (double)__bfloat162float(tb);
   }
   __syncthreads();
 
-  // ---- inverse of T_hat by Gauss-Jordan with partial pivoting (Rm becomes the inverse); T_xvsh = inverse^T
-  for (int idx = tid; idx < D * D; idx += BT_THREADS) Rm[idx] = ((idx / D) == (idx % D)) ? 1.0 : 0.0;
-  __syncthreads();
-  for (int col = 0; col < D; ++col) {
-    if (tid == 0) {
-      int pr = col; double pv = fabs(Tm[col * D + col]);
-      for (int r = col + 1; r < D; ++r) if (fabs(Tm[r * D + col]) > pv) { pv = fabs(Tm[r * D + col]); pr = r; }
-      perm[0] = pr;
-      if (!(pv > 0.0)) fail = 3;
-    }
-    __syncthreads();
-    const int pr = perm[0];
-    if (pr != col) {
-      for (int k = tid; k < D; k += BT_THREADS) {
-        double t = Tm[col * D + k]; Tm[col * D + k] = Tm[pr * D + k]; Tm[pr * D + k] = t;
-        t = Rm[col * D + k]; Rm[col * D + k] = Rm[pr * D + k]; Rm[pr * D + k] = t;
-      }
-    }
-    __syncthreads();
-    const double piv = Tm[col * D + col];
-    __syncthreads();
-    for (int k = tid; k < D; k += BT_THREADS) { Tm[col * D + k] /= piv; Rm[col * D + k] /= piv; }
-    __syncthreads();
-    // eliminate column `col` from every other row; factors are read before any row is modified
-    {
-      double* fac = Bm;                       // reuse: D factors
-      for (int r = tid; r < D; r += BT_THREADS) fac[r] = (r == col) ? 0.0 : Tm[r * D + col];
-      __syncthreads();
-      for (int idx = tid; idx < D * D; idx += BT_THREADS) {
-        const int r = idx / D, k = idx % D;
-        const double f = fac[r];
-        if (f != 0.0) { Tm[idx] -= f * Tm[col * D + k]; Rm[idx] -= f * Rm[col * D + k]; }
-      }
-    }
-    __syncthreads();
-  }
-  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
-    const int j = idx / D, k = idx % D;
-    Tinv_out[(size_t)c * D * D + idx] = (float)Rm[k * D + j];      // transpose of the inverse
-  }
+  inverse_transpose<D>(Tm, Rm, Bm, perm, &fail, Tinv_out + (size_t)c * D * D);
   if (tid == 0 && info != nullptr) info[c] = fail;
 }
 
+// (T)^-T of given bf16 transforms (Eq. 6 for transforms that were not built here)
+template <int D>
+__global__ void __launch_bounds__(BT_THREADS)
+invert_transforms_kernel(const __nv_bfloat16* __restrict__ T, float* __restrict__ Tinv_out, int32_t* __restrict__ info) {
+  extern __shared__ double sm[];
+  double* Tm = sm;
+  double* Rm = Tm + D * D;
+  double* fac = Rm + D * D;
+  __shared__ int perm[D];
+  __shared__ int fail;
+  const int c = blockIdx.x, tid = threadIdx.x;
+  if (tid == 0) fail = 0;
+  for (int idx = tid; idx < D * D; idx += BT_THREADS) Tm[idx] = (double)__bfloat162float(T[(size_t)c * D * D + idx]);
+  __syncthreads();
+  inverse_transpose<D>(Tm, Rm, fac, perm, &fail, Tinv_out + (size_t)c * D * D);
+  __syncthreads();
+  if (tid == 0 && info != nullptr) info[c] = fail;
+}
+
+cudaError_t run_invert_transforms(const void* T, int64_t K, int g, float* Tinv, int32_t* info, cudaStream_t st) {
+  const int C = (int)(K / g);
+  const size_t smem = (2 * (size_t)g * g + g) * sizeof(double);          // <= 16.6 KB: no attribute needed
+  const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
+  if (g == 32) invert_transforms_kernel<32><<<C, BT_THREADS, smem, st>>>(Tb, Tinv, info);
+  else invert_transforms_kernel<16><<<C, BT_THREADS, smem, st>>>(Tb, Tinv, info);
+  return cudaGetLastError();
+}
+
 cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* mom_x, int64_t n_x, int64_t K, int g,
-                                 double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st) {
+                                 double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st, bool with_hadamard) {
+  const int wh = with_hadamard ? 1 : 0;
   const int C = (int)(K / g);
   const size_t smem = 6 * (size_t)g * g * sizeof(double);
   __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(T);
@@ -240,9 +281,9 @@ cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* m
       if (e != cudaSuccess) return e;
       done = true;
     }
-    build_transforms_kernel<32><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info);
+    build_transforms_kernel<32><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info, wh);
   } else {
-    build_transforms_kernel<16><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info);
+    build_transforms_kernel<16><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info, wh);
   }
   return cudaGetLastError();
 }

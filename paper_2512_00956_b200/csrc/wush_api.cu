@@ -232,14 +232,30 @@ int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* momen
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
-int wush_build_transforms(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x, int64_t K, int g,
-                          float lambda, void* T, float* Tinv, int32_t* info, void* stream) {
+int wush_build_transforms_kind(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x, int64_t K,
+                               int g, float lambda, wush_transform_kind_t kind, void* T, float* Tinv, int32_t* info,
+                               void* stream) {
   if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  if (kind != WUSH_KIND_WUSH && kind != WUSH_KIND_WUS) return WUSH_ERR_FORMAT;
   if (K <= 0 || K % g != 0 || rows_w <= 0 || rows_x <= 0 || !(lambda >= 0.0f)) return WUSH_ERR_SHAPE;
   if (!mom_w || !mom_x || !T || !Tinv) return WUSH_ERR_NULL;
   if (!aligned16(mom_w) || !aligned16(mom_x) || !aligned16(T) || !aligned16(Tinv)) return WUSH_ERR_ALIGN;
   cudaError_t e = wush::run_build_transforms(mom_w, rows_w, mom_x, rows_x, K, g, (double)lambda, T, Tinv, info,
-                                             (cudaStream_t)stream);
+                                             (cudaStream_t)stream, kind == WUSH_KIND_WUSH);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
+int wush_build_transforms(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x, int64_t K, int g,
+                          float lambda, void* T, float* Tinv, int32_t* info, void* stream) {
+  return wush_build_transforms_kind(mom_w, rows_w, mom_x, rows_x, K, g, lambda, WUSH_KIND_WUSH, T, Tinv, info, stream);
+}
+
+int wush_invert_transforms(const void* T, int64_t K, int g, float* Tinv, int32_t* info, void* stream) {
+  if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  if (K <= 0 || K % g != 0) return WUSH_ERR_SHAPE;
+  if (!T || !Tinv) return WUSH_ERR_NULL;
+  if (!aligned16(T) || !aligned16(Tinv)) return WUSH_ERR_ALIGN;
+  cudaError_t e = wush::run_invert_transforms(T, K, g, Tinv, info, (cudaStream_t)stream);
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 

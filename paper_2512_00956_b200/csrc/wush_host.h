@@ -63,7 +63,9 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
                          const char** why);
 
 cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* mom_x, int64_t n_x, int64_t K, int g,
-                                 double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st);
+                                 double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st,
+                                 bool with_hadamard = true);
+cudaError_t run_invert_transforms(const void* T, int64_t K, int g, float* Tinv, int32_t* info, cudaStream_t st);
 
 // two-CTA persistent variant (M > 128); cudaErrorNotSupported = use the single-CTA kernel
 int gemm_2cta_cluster_limit(int clusters);   // test hook: 0 = no limit; returns the previous value (per device)

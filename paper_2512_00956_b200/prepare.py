@@ -2,9 +2,9 @@
 
 Second moments come from the library's calibration kernel (`wush_calib_moments`), the d x d
 factorisations of Algorithm 1 and the inverse-transpose of Eq. 6 from `wush_build_transforms`,
-the weight quantisation from `wush_quantize_weight`: nothing leaves the device.
-`build_transforms` below is the same construction written with torch.linalg; it is kept as an
-independent cross-check of the kernel and is not used by `QuantizedLinear`.
+the weight quantisation from `wush_quantize_weight`: nothing leaves the device.  The comparison
+transforms of Sec. 5 / Table 1 (one shared Hadamard matrix, the identity, WUSH without its Hadamard
+factor) go through the same calls; their weight-side partners come from `wush_invert_transforms`.
 
 Conventions (the paper leaves them open): damping ratio lambda = 0.01; singular values
 descending and each row of U^T W'^T signed so that its largest-magnitude entry is positive
@@ -28,31 +28,6 @@ def hadamard(d, device):
     return torch.where(pop % 2 == 0, 1.0, -1.0).to(torch.float64) / math.sqrt(d)
 
 
-def build_transforms(mom_w, n_w, mom_x, n_x, lam=0.01):
-    """Unnormalised moment sums [C,d,d] (fp32) + row counts -> (T bf16 [C,d,d], Tinv fp32 [C,d,d])."""
-    C, d, _ = mom_w.shape
-    dev = mom_w.device
-    eye = torch.eye(d, dtype=torch.float64, device=dev)
-    Mw = mom_w.to(torch.float64) / float(n_w)
-    Mx = mom_x.to(torch.float64) / float(n_x)
-    Mw = 0.5 * (Mw + Mw.transpose(1, 2))
-    Mx = 0.5 * (Mx + Mx.transpose(1, 2))
-    tr_w = torch.diagonal(Mw, dim1=1, dim2=2).sum(-1)
-    tr_x = torch.diagonal(Mx, dim1=1, dim2=2).sum(-1)
-    Wp = torch.linalg.cholesky(Mw + (lam * tr_w / d)[:, None, None] * eye)      # W' W'^T = damped M_W
-    Xp = torch.linalg.cholesky(Mx + (lam * tr_x / d)[:, None, None] * eye)
-    U, S, _ = torch.linalg.svd(Wp.transpose(1, 2) @ Xp)                         # W'^T X' = U S V^T
-    UtWt = U.transpose(1, 2) @ Wp.transpose(1, 2)
-    pick = UtWt.abs().argmax(dim=2, keepdim=True)
-    sgn = torch.sign(torch.gather(UtWt, 2, pick))
-    sgn = torch.where(sgn == 0, torch.ones_like(sgn), sgn)
-    UtWt = UtWt * sgn
-    T = hadamard(d, dev) @ (UtWt / torch.sqrt(S)[:, :, None])                   # H S^-1/2 U^T W'^T
-    T_bf16 = T.to(torch.bfloat16)
-    Tinv = torch.linalg.inv(T_bf16.to(torch.float64)).transpose(1, 2)           # T_xvsh = T^-T (Eq. 6)
-    return T_bf16.contiguous(), Tinv.to(torch.float32).contiguous()
-
-
 def fixed_transforms(kind, C, d, device):
     """The data-independent comparison transforms of Sec. 5 / Table 1, in the layout the kernels take:
     "hadamard" (the same normalised Hadamard matrix for every block, the H + Quant baseline) or
@@ -64,9 +39,11 @@ def fixed_transforms(kind, C, d, device):
         T1 = torch.eye(d, dtype=torch.float64, device=device)
     else:
         raise ValueError(kind)
-    T_bf16 = T1.to(torch.bfloat16)
-    Tinv = torch.linalg.inv(T_bf16.to(torch.float64)).transpose(0, 1).to(torch.float32)
-    return T_bf16.expand(C, d, d).contiguous(), Tinv.expand(C, d, d).contiguous()
+    T = T1.to(torch.bfloat16).expand(C, d, d).contiguous()
+    Tinv, info = wush.invert_transforms(T, d)                                    # Eq. 6 for the stored values
+    if int(info.abs().max().item()) != 0:
+        raise wush.WushError("wush_invert_transforms: singular transform")
+    return T, Tinv
 
 
 class QuantizedLinear:
@@ -76,12 +53,12 @@ class QuantizedLinear:
         f, g = wush.FORMATS[fmt]
         self.fmt, self.g = fmt, g
         self.N, self.K = W.shape
-        if transform == "wush":
+        if transform in ("wush", "wus"):
             mom_w, cnt_w = wush.calib_moments(W, g)
             mom_x, cnt_x = wush.calib_moments(Xc, g)
             # Algorithm 1 + Eq. 6 for every block in the library's own kernel (fp64 Cholesky, Jacobi SVD)
             self.T, self.Tinv, self.info = wush.build_transforms(mom_w, int(cnt_w[0].item()), mom_x,
-                                                                 int(cnt_x[0].item()), g, lam)
+                                                                 int(cnt_x[0].item()), g, lam, kind=transform)
             if int(self.info.abs().max().item()) != 0:
                 raise wush.WushError("wush_build_transforms: a block failed to factorise (see info)")
         else:

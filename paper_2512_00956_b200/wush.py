@@ -26,7 +26,7 @@ EXPORTS = [
     "wush_linear_workspace_bytes", "wush_calib_moments", "wush_calib_moments_workspace_bytes",
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
     "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division", "wush_debug_gemm_clusters",
-    "wush_debug_drop_tile", "wush_decode_status",
+    "wush_debug_drop_tile", "wush_decode_status", "wush_build_transforms_kind", "wush_invert_transforms",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -64,6 +64,8 @@ def lib():
         L.wush_calib_moments_workspace_bytes.argtypes = [i64, i64, i32]
         L.wush_build_transforms.argtypes = [vp, i64, vp, i64, i64, i32, ctypes.c_float, vp, vp, vp, vp]
         L.wush_build_transforms.restype = i32
+        L.wush_build_transforms_kind.argtypes = [vp, i64, vp, i64, i64, i32, ctypes.c_float, i32, vp, vp, vp, vp]
+        L.wush_invert_transforms.argtypes = [vp, i64, i32, vp, vp, vp]
         L.wush_calib_moments_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]
         L.wush_debug_gemm_clusters.argtypes = [i32]
         L.wush_debug_gemm_clusters.restype = i32
@@ -227,17 +229,31 @@ def calib_moments(Xc, g, moments=None, count=None, workspace=None):
     return moments, count
 
 
-def build_transforms(mom_w, rows_w, mom_x, rows_x, g, lam=0.01):
-    """Moment sums fp32 [K/g,g,g] (+ row counts) -> (T bf16 [K/g,g,g], Tinv fp32 [K/g,g,g], info int32 [K/g])."""
+KINDS = {"wush": 0, "wus": 1}
+
+
+def build_transforms(mom_w, rows_w, mom_x, rows_x, g, lam=0.01, kind="wush"):
+    """Moment sums fp32 [K/g,g,g] (+ row counts) -> (T bf16 [K/g,g,g], Tinv fp32 [K/g,g,g], info int32 [K/g]).
+    kind "wus" leaves the Hadamard factor out (the ablation of Table 1)."""
     _dev(mom_w, mom_x)
     C = mom_w.shape[0]
     K = C * g
     T = torch.empty((C, g, g), dtype=torch.bfloat16, device=mom_w.device)
     Tinv = torch.empty((C, g, g), dtype=torch.float32, device=mom_w.device)
     info = torch.zeros(max(C, 4), dtype=torch.int32, device=mom_w.device)
-    check(lib().wush_build_transforms(_ptr(mom_w), int(rows_w), _ptr(mom_x), int(rows_x), K, g, float(lam), _ptr(T),
-                                      _ptr(Tinv), _ptr(info), _stream()))
+    check(lib().wush_build_transforms_kind(_ptr(mom_w), int(rows_w), _ptr(mom_x), int(rows_x), K, g, float(lam),
+                                           KINDS[kind], _ptr(T), _ptr(Tinv), _ptr(info), _stream()))
     return T, Tinv, info[:C]
+
+
+def invert_transforms(T, g):
+    """T bf16 [K/g,g,g] -> (Tinv fp32 [K/g,g,g] = T^-T per block, info int32 [K/g])."""
+    _dev(T)
+    C = T.shape[0]
+    Tinv = torch.empty((C, g, g), dtype=torch.float32, device=T.device)
+    info = torch.zeros(max(C, 4), dtype=torch.int32, device=T.device)
+    check(lib().wush_invert_transforms(_ptr(T), C * g, g, _ptr(Tinv), _ptr(info), _stream()))
+    return Tinv, info[:C]
 
 
 def calib_moments_static(Xc, g, moments=None, count=None):

@@ -245,10 +245,10 @@ def test_linear_bf16_output_config2_bench_configuration():
     assert rel_fro(Y.float().cpu().numpy(), Yo) <= 1e-3
 
 
-@pytest.mark.parametrize("kind", ["hadamard", "identity"])
+@pytest.mark.parametrize("kind", ["hadamard", "identity", "wus"])
 def test_fixed_transform_variants_run_through_the_same_kernels(kind):
-    """H + Quant and None + Quant (Sec. 5) are the WUSH kernels with a replicated / identity T; on a layer
-    with outlier channels the ordering of Table 1 must show: WUSH < Hadamard < identity (MXFP4)."""
+    """H + Quant, None + Quant (Sec. 5) and WUS (Table 1) are the WUSH kernels with another T; on a layer
+    with outlier channels the ordering of Table 1 must show: WUSH below each of them (MXFP4)."""
     from paper_2512_00956_b200 import prepare
     cfg = synth.CONFIGS[1]
     d = synth.layer_inputs(cfg, M=128, N=256, K=512, B=512)
@@ -306,3 +306,39 @@ def test_build_transforms_kernel_against_oracle_and_identities(fmt, K):
     Y0 = F.bf16_bits_to_f64(d["X"]) @ Wv.T
     lg, lo = rel_fro(Y.cpu().numpy(), Y0), rel_fro(L.forward(d["X"]), Y0)
     assert abs(lg - lo) <= 0.15 * lo, (lg, lo)
+
+
+@pytest.mark.parametrize("g,K", [(32, 512), (16, 256)])
+def test_wus_kind_and_invert_transforms(g, K):
+    """WUSH_KIND_WUS is WUSH without its Hadamard factor (Table 1's "WUS"): H T_wus reproduces the WUSH transform
+    of the same moments, and the kernel agrees with the oracle's WUS; wush_invert_transforms returns the
+    inverse-transpose of any stored transforms (Eq. 6)."""
+    from oracle import wush_transform as WT
+    cfg = synth.CONFIGS[1]
+    d = synth.layer_inputs(cfg, M=16, N=512, K=K, B=512)
+    Wv, Xcv = F.bf16_bits_to_f64(d["W"]), F.bf16_bits_to_f64(d["Xc"])
+    sW, sX = P.second_moment_sums(Wv, g), P.second_moment_sums(Xcv, g)
+    args = (dev(sW.astype(np.float32)), Wv.shape[0], dev(sX.astype(np.float32)), Xcv.shape[0], g, 0.01)
+    Tw, _, info_w = wush.build_transforms(*args)
+    Ts, Tsinv, info_s = wush.build_transforms(*args, kind="wus")
+    _sync()
+    assert int(info_w.abs().max().item()) == 0 and int(info_s.abs().max().item()) == 0
+    Tw, Ts, Tsinv = Tw.double().cpu().numpy(), Ts.double().cpu().numpy(), Tsinv.double().cpu().numpy()
+    H = WT.hadamard(g)
+    C = K // g
+    for c in range(C):
+        scale = np.abs(Tw[c]).max()
+        assert np.allclose(H @ Ts[c], Tw[c], atol=2.0 ** -6 * scale * np.sqrt(g))     # two bf16 roundings apart
+        assert np.allclose(Tsinv[c] @ Ts[c].T, np.eye(g), atol=1e-5)                  # Eq. 6 on the stored values
+        To = WT.variant_transform("WUS", sW[c] / Wv.shape[0], sX[c] / Xcv.shape[0], 0.01)
+        assert np.allclose(Ts[c], To, atol=2.0 ** -7 * np.abs(To).max() + 1e-12, rtol=2.0 ** -7)
+    # inverse-transpose of arbitrary (here: random, well conditioned) bf16 transforms
+    rng = np.random.default_rng(g)
+    A = np.eye(g)[None] + 0.2 * rng.standard_normal((C, g, g))
+    Ab = F.f64_to_bf16_bits(A)
+    Tinv, info = wush.invert_transforms(dev_bf16(Ab), g)
+    _sync()
+    assert int(info.abs().max().item()) == 0
+    Av = F.bf16_bits_to_f64(Ab)
+    ref = np.stack([np.linalg.inv(Av[c]).T for c in range(C)])
+    assert np.allclose(Tinv.double().cpu().numpy(), ref, rtol=1e-5, atol=1e-6)
