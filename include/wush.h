@@ -124,6 +124,13 @@ int wush_quantize_act_dynamic(const void* X, int64_t M, int64_t K, const void* T
                               float* x_tensor_scale, uint8_t* codes, uint8_t* scales,
                               wush_sf_layout_t sf, void* stream);
 
+/* The static NVFP4 activation tensor scale from calibration tokens (offline): the AbsMax pass of the call
+ * above on Xc bf16 [B,K], without quantising.  out fp32[2] on the device, 8-byte aligned, WRITTEN:
+ * [0] = AbsMax / (6 * 448) (1 if everything is zero), [1] = the AbsMax over all B x K transformed values.
+ * g must be 16, B >= 1.  Errors: NULL / SHAPE / FORMAT / ALIGN / CUDA. */
+int wush_act_tensor_scale(const void* Xc, int64_t B, int64_t K, const void* T, int g, float* out,
+                          void* stream);
+
 /* Offline weight preparation (Algorithm 2, RTN case, last line):
  *   W~ = q( W_blk * Tinv_c^T ),  Tinv = T_xvsh = T_wush^-T (Eq. 6) given in fp32.
  *   W      bf16 [N,K];  Tinv fp32 [K/g][g][g] (same index convention as T above).

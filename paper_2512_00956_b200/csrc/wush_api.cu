@@ -124,6 +124,17 @@ int wush_quantize_act_dynamic(const void* X, int64_t M, int64_t K, const void* T
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 
+int wush_act_tensor_scale(const void* Xc, int64_t B, int64_t K, const void* T, int g, float* out, void* stream) {
+  int rc = check_fmt(WUSH_NVFP4, g);
+  if (rc) return rc;
+  if ((rc = check_shape(B, K, g))) return rc;
+  if (!Xc || !T || !out) return WUSH_ERR_NULL;
+  if (!aligned16(Xc) || !aligned16(T) || (reinterpret_cast<uintptr_t>(out) & 7u) != 0) return WUSH_ERR_ALIGN;
+  if (B == 0) return WUSH_ERR_SHAPE;
+  const cudaError_t e = wush::run_act_tensor_scale(Xc, B, K, T, out, (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
 size_t wush_quantize_weight_workspace_bytes(int64_t, int64_t, wush_format_t, int) { return 256; }
 
 int wush_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv, wush_format_t fmt, int g,

@@ -30,6 +30,8 @@ cudaError_t run_quantize_act(const void* X, int64_t M, int64_t K, const void* T,
                              uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
                              bool pdl, cudaStream_t st, const QuantOpts& opt = QuantOpts());
 cudaError_t run_act_amax(const void* X, int64_t M, int64_t K, const void* T, uint32_t* amax, cudaStream_t st);
+// out[0] = NVFP4 tensor scale of the transformed tokens (AbsMax / 2688, 1 if all zero), out[1] = that AbsMax
+cudaError_t run_act_tensor_scale(const void* X, int64_t M, int64_t K, const void* T, float* out, cudaStream_t st);
 // streaming (TMA-fed, persistent) variant; cudaErrorNotSupported = problem not covered, use the other kernel
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                     uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,

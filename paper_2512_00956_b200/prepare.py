@@ -65,8 +65,7 @@ class QuantizedLinear:
             self.T, self.Tinv = fixed_transforms(transform, self.K // g, g, W.device)
         self.w_codes, self.w_scales, self.w_tensor_scale = wush.quantize_weight(W, self.Tinv, fmt, sf=wush.SF_TILED)
         if fmt == "nvfp4":
-            v = wush.transform_act_f32(Xc, self.T, g)                            # static activation tensor scale
-            self.x_tensor_scale = (v.abs().max().to(torch.float32) / 2688.0).reshape(1).repeat(4).contiguous()
+            self.x_tensor_scale = wush.act_tensor_scale(Xc, self.T, g)          # static: from the calibration tokens
         else:
             self.x_tensor_scale = None
         self._ws = None

@@ -27,6 +27,7 @@ EXPORTS = [
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
     "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division", "wush_debug_gemm_clusters",
     "wush_debug_drop_tile", "wush_decode_status", "wush_build_transforms_kind", "wush_invert_transforms",
+    "wush_act_tensor_scale",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -66,6 +67,7 @@ def lib():
         L.wush_build_transforms.restype = i32
         L.wush_build_transforms_kind.argtypes = [vp, i64, vp, i64, i64, i32, ctypes.c_float, i32, vp, vp, vp, vp]
         L.wush_invert_transforms.argtypes = [vp, i64, i32, vp, vp, vp]
+        L.wush_act_tensor_scale.argtypes = [vp, i64, i64, vp, i32, vp, vp]
         L.wush_calib_moments_static.argtypes = [vp, i64, i64, i32, vp, vp, vp]
         L.wush_debug_gemm_clusters.argtypes = [i32]
         L.wush_debug_gemm_clusters.restype = i32
@@ -144,6 +146,14 @@ def quantize_act_dynamic(X, T, sf=SF_LINEAR, out=None, x_tensor_scale=None):
     ts = x_tensor_scale if x_tensor_scale is not None else torch.zeros(4, dtype=torch.float32, device=X.device)
     check(lib().wush_quantize_act_dynamic(_ptr(X), M, K, _ptr(T), 16, _ptr(ts), _ptr(codes), _ptr(scales), sf, _stream()))
     return codes, scales, ts
+
+
+def act_tensor_scale(Xc, T, g=16):
+    """Static NVFP4 activation tensor scale of calibration tokens: fp32[4] on the device, [0] = scale, [1] = AbsMax."""
+    _dev(Xc, T)
+    out = torch.zeros(4, dtype=torch.float32, device=Xc.device)
+    check(lib().wush_act_tensor_scale(_ptr(Xc), Xc.shape[0], Xc.shape[1], _ptr(T), g, _ptr(out), _stream()))
+    return out
 
 
 def quantize_weight(W, Tinv, fmt, sf=SF_TILED, out=None):

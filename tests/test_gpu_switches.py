@@ -148,6 +148,17 @@ def test_branch_free_division_equals_ieee_division_for_every_x():
     assert int(bad.abs().max().item()) == 0, [(float(divs[i]), int(b)) for i, b in enumerate(bad.cpu().tolist()) if b]
 
 
+def test_static_tensor_scale_of_calibration_tokens():
+    """wush_act_tensor_scale: AbsMax of the transformed calibration tokens within the transform's tolerance of
+    the oracle's, and the scale is exactly that AbsMax / 2688 in fp32 - the oracle's static ts_x."""
+    d, L = _layer(1, "nvfp4", M=16, N=256, K=1024, B=700)
+    out = wush.act_tensor_scale(dev_bf16(d["Xc"]), dev_bf16(L.T_bits), 16).cpu().numpy()
+    amax_o = np.float32(L.ts_x) * np.float32(2688.0)
+    assert abs(out[1] - amax_o) <= 1e-5 * amax_o
+    assert out[0] == np.float32(out[1]) / np.float32(2688.0)
+    assert abs(out[0] - L.ts_x) <= 1e-5 * L.ts_x
+
+
 # ------------------------------------------------------------------ error path: a bounded wait that runs out
 def test_expired_wait_is_reported_and_the_next_call_works():
     """The test hook leaves one tile of the quantiser unrequested: the consumers' bounded wait for it
