@@ -59,3 +59,20 @@ def test_result_does_not_depend_on_the_number_of_clusters(fmt, M, N, K):
             assert torch.equal(Yb, Y0b), f"bf16 output changed with {limit} clusters"
     finally:
         wush.debug_gemm_clusters(old)
+
+
+@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4"])
+@pytest.mark.parametrize("M,N,K", [(129, 8, 64), (130, 24, 192), (257, 264, 320), (513, 40, 576)])
+def test_smallest_and_ragged_shapes_of_the_two_cta_path(fmt, M, N, K):
+    """M just above the single-CTA limit, N of a few columns, K of one partial slab (64, 192) or of a whole
+    slab plus a partial one (320, 576): against the fp64 oracle product of the same codes."""
+    rng = np.random.default_rng(M + N + K)
+    xc, xs = _operand(rng, M, K, fmt)
+    wc, ws = _operand(rng, N, K, fmt)
+    ts = 0.031 if fmt == "nvfp4" else None
+    tsd = dev(np.full(4, ts, dtype=np.float32)) if fmt == "nvfp4" else None
+    Y, st = wush.gemm_fp4(dev(F.pack_e2m1(xc)), dev(tile(xs)), dev(F.pack_e2m1(wc)), dev(tile(ws)), K, fmt, tsd, tsd)
+    torch.cuda.synchronize()
+    assert int(st[0].item()) == 0
+    Yo = P.dequantized_product(Q.dequantize(xc, xs, fmt, ts), Q.dequantize(wc, ws, fmt, ts))
+    assert rel_fro(Y.cpu().numpy(), Yo) <= 1e-5
