@@ -28,6 +28,18 @@ def test_exports_match_header(L):
     assert declared >= set(wush.EXPORTS)
 
 
+def test_header_is_plain_c_and_cpp(tmp_path):
+    """include/wush.h is the boundary: it must compile on its own as C99 and as C++ (no torch, no CUDA types)."""
+    import shutil
+    import subprocess
+    hdr = os.path.join(ROOT, "include", "wush.h")
+    for cc, flags in (("gcc", ["-std=c99", "-pedantic", "-x", "c"]), ("g++", ["-std=c++11", "-x", "c++"])):
+        if shutil.which(cc) is None:
+            pytest.skip(f"{cc} not installed")
+        res = subprocess.run([cc, "-Wall", "-Werror", "-fsyntax-only"] + flags + [hdr], capture_output=True, text=True)
+        assert res.returncode == 0, res.stderr
+
+
 def test_status_strings(L):
     assert L.wush_status_string(0) == b"ok"
     for code in range(-8, 0):
