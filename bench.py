@@ -1,20 +1,28 @@
 #!/usr/bin/env python
 """Benchmark of the online W4A4 WUSH linear layer (Eq. 7) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 5] [--m 16384] [--impl ours|reference]
 
 A step is one pass of the whole hot path - fused transform + quantise of X, then the
 block-scaled FP4 GEMM against the pre-quantised weights - over one batch of synthetic tokens
 (`wush_linear`).  Rank 0 prints ONE JSON line.  `value` is 2*M*N*K / step time summed over
 ranks (each rank runs its own replica of the layer on its own tokens: weak scaling, no
-data-path collective).  The line also carries the roofline of the dominant kernel, the
-quantiser's HBM figure, the cuBLAS bf16 GEMM of the same shape, an end-to-end number with
-host buffers, sampled clocks, and the CPU oracle timed on the host cores.
+data-path collective).  The default workload is the largest single-GPU one: the Llama-3.1-70B
+MLP shape (K = 8192, N = 28672) at 16384 tokens, MXFP4.
+
+Timing: the K steps are captured once in a CUDA graph; the graph is replayed R times between
+CUDA events (R chosen so that the replays cover at least 50 ms), and the median replay gives the
+step time.  The same protocol times the two kernels of the step alone, the cuBLAS bf16 GEMM and
+the library's own block-scaled FP4 GEMM of the same shape.  The line also carries the roofline
+of the dominant kernel, the quantiser's HBM figure, an end-to-end number with host buffers,
+sampled clocks, the CPU oracle timed on the host cores, and a `workloads` array with the other
+benchmark shapes measured the same way.
 
 `--impl reference` times the CPU oracle (the only "reference" this method has here).
 """
 import argparse
 import json
+import math
 import os
 import statistics
 import sys
@@ -25,6 +33,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "W4A4 WUSH linear TFLOP/s (2MNK / step time; transform+quant + FP4 GEMM)"
+MIN_TIMED_MS = 50.0            # replays of the headline graph cover at least this much device time
+MIN_TIMED_MS_SIDE = 20.0       # per-kernel graphs and the `workloads` entries
+FP4_SPEC_TFLOPS = 9000.0       # vendor's dense FP4 figure, reported beside the measured ceilings
+HBM_SPEC_GBS = 8000.0
 
 
 def load_peaks():
@@ -83,15 +95,31 @@ class ClockSampler:
         if self._thread is not None:
             self._thread.join(timeout=2)
         med = statistics.median(self.samples) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "sm_mhz_min": min(self.samples) if self.samples else None}
 
 
 def pick_config(args):
     from paper_2512_00956_b200 import synth
     cfg = synth.CONFIGS[args.config]
     fmt = args.fmt or cfg.formats[0]
-    M = args.m or cfg.M
+    if args.m is not None:
+        M = args.m
+    elif cfg.m_sweep:
+        M = max(cfg.m_sweep)                 # the token sweep's largest point: the prefill end of the regime
+    else:
+        M = cfg.M
     return cfg, fmt, M
+
+
+def config_of(args, cfg, fmt, M):
+    """The `config` object of the JSON line - the same for both arms, so that their lines are comparable."""
+    from paper_2512_00956_b200 import synth
+    dyn = bool(args.dynamic_ts and fmt == "nvfp4")
+    return {"workload": cfg.name, "M": M, "K": cfg.K, "N": cfg.N, "format": fmt, "g": synth.GROUP[fmt],
+            "y_dtype": args.out, "transform": args.transform,
+            "x_tensor_scale": ("per batch" if dyn else "static") if fmt == "nvfp4" else None, "tokens_per_rank": M,
+            "l2": "GPU arm: every step works on its own rotating copy of X, workspace, Y and W~ (copies together > 2x L2)"}
 
 
 def oracle_sample_seconds(cfg, fmt, M, rows, dynamic=False, budget_s=12.0):
@@ -144,17 +172,174 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": tf, "unit": "TFLOP/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "M": M, "K": cfg.K, "N": cfg.N, "format": fmt, "sample_rows": rows},
+            "config": config_of(args, cfg, fmt, M), "sample_rows": rows,
             "cpu_baseline": {"value": tf, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": tf, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+class Workload:
+    """One layer shape on one GPU: prepared weights, rotating cold buffer sets, and the launches to time."""
+
+    def __init__(self, cfg, fmt, M, dev, out, transform="wush", dynamic=False, W=None, Xc=None):
+        import numpy as np
+        import torch
+        from paper_2512_00956_b200 import prepare, synth, wush
+        self.torch, self.wush = torch, wush
+        self.cfg, self.fmt, self.M, self.dev, self.out = cfg, fmt, M, dev, out
+        self.g = g = synth.GROUP[fmt]
+        self.K, self.N = K, N = cfg.K, cfg.N
+        self.out_dtype = torch.bfloat16 if out == "bf16" else torch.float32
+
+        def up(bits):
+            return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(dev)
+
+        self.Xh_bits = synth.activations(cfg, M=M)
+        self.W = W if W is not None else up(synth.weights(cfg))
+        self.Xc = Xc if Xc is not None else up(synth.calibration(cfg))
+        self.layer = layer = prepare.QuantizedLinear(self.W, self.Xc, fmt, transform=transform)
+        X0 = up(self.Xh_bits)
+        self.ws_bytes = ws_bytes = wush.linear_workspace_bytes(M, K, g)
+        # buffer rotation: every step works on its own copy of X, workspace, Y and of the quantised weights,
+        # and the copies together exceed twice the L2 capacity, so each step's data is cold while the (tiny)
+        # kernel code stays warm
+        ybytes = 2 if out == "bf16" else 4
+        self.set_bytes = X0.numel() * 2 + ws_bytes + M * N * ybytes + layer.w_codes.numel() + layer.w_scales.numel()
+        self.nsets = nsets = max(2, int((2 * 126e6) // self.set_bytes) + 2)
+        self.sets = []
+        for i in range(nsets):
+            d_ = dict(X=X0 if i == 0 else X0.clone(), Y=torch.empty((M, N), dtype=self.out_dtype, device=dev),
+                      ws=torch.empty(ws_bytes, dtype=torch.uint8, device=dev),
+                      wq=layer.w_codes if i == 0 else layer.w_codes.clone(),
+                      wsc=layer.w_scales if i == 0 else layer.w_scales.clone(),
+                      status=torch.zeros(4, dtype=torch.int32, device=dev))
+            d_["xq"] = d_["ws"][: M * K // 2].view(M, K // 2)
+            d_["xs"] = d_["ws"][(M * K // 2 + 15) // 16 * 16:][: wush.scale_bytes(M, K, g, wush.SF_TILED)]
+            self.sets.append(d_)
+        self.dynamic = bool(dynamic and fmt == "nvfp4")
+        self.ts_step = None if self.dynamic else layer.x_tensor_scale   # None: wush_linear finds the scale of each batch itself
+        self.ts_buf = torch.zeros(4, dtype=torch.float32, device=dev)
+        self.flops = 2.0 * M * N * K
+        self.q_bytes = 2.0 * M * K + M * K / 2.0 + M * K / g + 2.0 * K * g
+        self.g_bytes = M * K / 2.0 + M * K / g + N * K / 2.0 + N * K / g + M * N * ybytes
+
+    def step(self, d_):
+        L = self.layer
+        self.wush.linear(d_["X"], L.T, d_["wq"], d_["wsc"], self.fmt, self.ts_step, L.w_tensor_scale,
+                         out=d_["Y"], workspace=d_["ws"])
+
+    def quant_only(self, d_):
+        L, w = self.layer, self.wush
+        if self.dynamic:
+            w.quantize_act_dynamic(d_["X"], L.T, w.SF_TILED, out=(d_["xq"], d_["xs"]), x_tensor_scale=self.ts_buf)
+        else:
+            w.quantize_act(d_["X"], L.T, self.fmt, L.x_tensor_scale, w.SF_TILED, out=(d_["xq"], d_["xs"]))
+
+    def gemm_only(self, d_):
+        L = self.layer
+        self.wush.gemm_fp4(d_["xq"], d_["xs"], d_["wq"], d_["wsc"], self.K, self.fmt, L.x_tensor_scale, L.w_tensor_scale,
+                           out=d_["Y"], status=d_["status"])
+
+    def status(self):
+        return max(self.wush.linear_status(d_["ws"], self.M, self.K, self.g) for d_ in self.sets)
+
+    def release(self):
+        self.sets = None
+        self.layer = None
+        self.torch.cuda.empty_cache()
+
+
+def timed(fn, sets, steps, min_ms, dev, barrier=None, what="step"):
+    """`steps` launches of fn over the rotating sets inside ONE CUDA graph; the graph is replayed R times, each
+    replay bracketed by CUDA events on the launching stream (pure device time, no per-launch host latency),
+    R chosen so that all replays together cover at least min_ms.  Returns (median ms per step, replays,
+    list of per-replay ms per step, graph used).  Falls back to an eager loop if capture fails."""
+    import torch
+    nsets = len(sets)
+    side = torch.cuda.Stream(device=dev)
+    graph = None
+    try:
+        with torch.cuda.stream(side):
+            for i in range(min(2, steps)):
+                fn(sets[i % nsets])
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(steps):
+                    fn(sets[i % nsets])
+    except Exception as exc:           # pragma: no cover
+        sys.stderr.write(f"[bench] CUDA-graph capture of {what} failed ({exc}); timing an eager loop\n")
+        graph = None
+        torch.cuda.synchronize()
+
+    def once():
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if barrier is not None:
+            side.synchronize()
+            barrier()
+        a.record(side)
+        if graph is not None:
+            graph.replay()
+        else:
+            for i in range(steps):
+                fn(sets[i % nsets])
+        b.record(side)
+        return a, b
+
+    with torch.cuda.stream(side):
+        a, b = once()                                        # untimed warm-up replay, also sizes R
+        side.synchronize()
+        est = max(a.elapsed_time(b), 1e-3)
+        replays = max(3, min(2000, int(math.ceil(min_ms / est))))
+        pairs = [once() for _ in range(replays)]
+        side.synchronize()
+    if barrier is not None:
+        barrier()
+    per = [x.elapsed_time(y) / steps for x, y in pairs]
+    return statistics.median(per), replays, per, graph is not None
+
+
+def library_fp4_gemm_ms(wl, steps, dev):
+    """cuBLASLt's block-scaled FP4 GEMM of the same shape through torch._scaled_mm on this workload's own codes
+    and scale bytes - context beside `bf16_gemm`, never on the product path.  None if torch cannot run it."""
+    import torch
+    try:
+        sdt = torch.float8_e8m0fnu if wl.g == 32 else torch.float8_e4m3fn
+
+        def fn(d_):
+            torch._scaled_mm(d_["xq"].view(torch.float4_e2m1fn_x2), d_["wq"].view(torch.float4_e2m1fn_x2).t(),
+                             d_["xs"].view(sdt), d_["wsc"].view(sdt), out_dtype=torch.bfloat16)
+        fn(wl.sets[0])
+        torch.cuda.synchronize()
+        ms, _, _, _ = timed(fn, wl.sets, steps, MIN_TIMED_MS_SIDE, dev, what="library fp4 gemm")
+        return ms
+    except Exception as exc:
+        sys.stderr.write(f"[bench] library FP4 GEMM not available: {str(exc)[:200]}\n")
+        return None
+
+
+def fractions(wl, peaks, step_ms, q_ms, g_ms):
+    """TFLOP/s, GB/s and the fractions of the measured and nominal ceilings for one workload."""
+    gemm_tf = wl.flops / (g_ms * 1e-3) / 1e12
+    q_gbs = wl.q_bytes / (q_ms * 1e-3) / 1e9
+    out = {"step_us": step_ms * 1e3, "gemm_us": g_ms * 1e3, "quant_us": q_ms * 1e3,
+           "step_tflops": wl.flops / (step_ms * 1e-3) / 1e12, "gemm_tflops": gemm_tf, "quant_gbs": q_gbs,
+           "quant_frac_of_measured_hbm": q_gbs / peaks["hbm_gbs"], "quant_frac_of_8tbs": q_gbs / HBM_SPEC_GBS}
+    if wl.M > 128:
+        out.update({"gemm_bound": "tensor", "gemm_frac_of_measured_burst_x4": gemm_tf / (4 * peaks["bf16_tflops"]),
+                    "gemm_frac_of_measured_sustained_x4": gemm_tf / (4 * peaks["bf16_tflops_sustained"]),
+                    "gemm_frac_of_9pf": gemm_tf / FP4_SPEC_TFLOPS})
+    else:
+        g_gbs = wl.g_bytes / (g_ms * 1e-3) / 1e9
+        out.update({"gemm_bound": "hbm", "gemm_gbs": g_gbs, "gemm_frac_of_measured_hbm": g_gbs / peaks["hbm_gbs"]})
+    return out
 
 
 def run_ours(args):
     import numpy as np
     import torch
     from paper_2512_00956_b200 import dist as D
-    from paper_2512_00956_b200 import prepare, synth, wush
+    from paper_2512_00956_b200 import synth, wush
 
     rank, local_rank, world = D.init()
     if not torch.cuda.is_available():
@@ -164,106 +349,30 @@ def run_ours(args):
     wush.lib()                                           # fail loudly if the library is missing
     peaks = load_peaks()
     cfg, fmt, M = pick_config(args)
-    g = synth.GROUP[fmt]
-    K, N = cfg.K, cfg.N
-    out_dtype = torch.bfloat16 if args.out == "bf16" else torch.float32
-
-    def up(bits):
-        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(dev)
-
-    Xh_bits = synth.activations(cfg, M=M)
-    W, Xc = up(synth.weights(cfg)), up(synth.calibration(cfg))
-    layer = prepare.QuantizedLinear(W, Xc, fmt, transform=args.transform)
-    X0 = up(Xh_bits)
-    ws_bytes = wush.linear_workspace_bytes(M, K, g)
+    wl = Workload(cfg, fmt, M, dev, args.out, args.transform, args.dynamic_ts)
+    g, K, N = wl.g, wl.K, wl.N
+    sets, nsets = wl.sets, wl.nsets
     stream = torch.cuda.current_stream()
-
-    # ---- buffer rotation: every step works on its own copy of X, workspace, Y and of the quantised
-    # weights, and the copies together exceed twice the L2 capacity, so each step's data is cold
-    # while the (tiny) kernel code stays warm.
-    set_bytes = X0.numel() * 2 + ws_bytes + M * N * (2 if args.out == "bf16" else 4) + layer.w_codes.numel() + layer.w_scales.numel()
-    nsets = max(2, int((2 * 126e6) // set_bytes) + 2)
-    sets = []
-    for i in range(nsets):
-        sets.append(dict(X=X0.clone(), Y=torch.empty((M, N), dtype=out_dtype, device=dev),
-                         ws=torch.empty(ws_bytes, dtype=torch.uint8, device=dev),
-                         wq=layer.w_codes.clone(), wsc=layer.w_scales.clone(),
-                         status=torch.zeros(4, dtype=torch.int32, device=dev)))
-    for d_ in sets:
-        d_["xq"] = d_["ws"][: M * K // 2].view(M, K // 2)
-        d_["xs"] = d_["ws"][(M * K // 2 + 15) // 16 * 16:][: wush.scale_bytes(M, K, g, wush.SF_TILED)]
-
-    dynamic = bool(args.dynamic_ts and fmt == "nvfp4")
-    ts_step = None if dynamic else layer.x_tensor_scale      # None: wush_linear finds the scale of each batch itself
-    ts_buf = torch.zeros(4, dtype=torch.float32, device=dev)
-
-    def step(d_):
-        wush.linear(d_["X"], layer.T, d_["wq"], d_["wsc"], fmt, ts_step, layer.w_tensor_scale,
-                    out=d_["Y"], workspace=d_["ws"])
-
-    def quant_only(d_):
-        if dynamic:
-            wush.quantize_act_dynamic(d_["X"], layer.T, wush.SF_TILED, out=(d_["xq"], d_["xs"]), x_tensor_scale=ts_buf)
-        else:
-            wush.quantize_act(d_["X"], layer.T, fmt, layer.x_tensor_scale, wush.SF_TILED, out=(d_["xq"], d_["xs"]))
-
-    def gemm_only(d_):
-        wush.gemm_fp4(d_["xq"], d_["xs"], d_["wq"], d_["wsc"], K, fmt, layer.x_tensor_scale, layer.w_tensor_scale,
-                      out=d_["Y"], status=d_["status"])
-
-    def timed(fn, steps, what):
-        """K launches of fn over the rotating sets inside ONE CUDA graph, bracketed by events on the launching
-        stream: pure device time, no per-launch host latency.  Falls back to an eager loop if capture fails."""
-        side = torch.cuda.Stream(device=dev)
-        graph = None
-        try:
-            with torch.cuda.stream(side):
-                for i in range(min(2, steps)):
-                    fn(sets[i % nsets])
-                side.synchronize()
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(graph, stream=side):
-                    for i in range(steps):
-                        fn(sets[i % nsets])
-        except Exception as exc:           # pragma: no cover
-            sys.stderr.write(f"[bench] CUDA-graph capture of {what} failed ({exc}); timing an eager loop\n")
-            graph = None
-            torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(side):
-            if graph is not None:
-                graph.replay()                                           # untimed warm-up replay
-            side.synchronize()
-            D.barrier()
-            a.record(side)
-            if graph is not None:
-                graph.replay()
-            else:
-                for i in range(steps):
-                    fn(sets[i % nsets])
-            b.record(side)
-            side.synchronize()
-        D.barrier()
-        return a.elapsed_time(b) / steps, graph is not None
-
-    for i in range(max(3, args.warmup)):
-        step(sets[i % nsets])
+    warm = max(3, args.warmup)
+    for i in range(warm):
+        wl.step(sets[i % nsets])
     torch.cuda.synchronize()
 
-    # ---- timed region: exactly K steps
+    # ---- timed region: graphs of exactly K steps, replayed; median replay, max over ranks
     sampler = ClockSampler(local_rank)
     sampler.start()
     wall0 = time.perf_counter()
-    ms_rank, used_graph = timed(step, args.steps, "step")
+    ms_rank, replays, per_replay, used_graph = timed(wl.step, sets, args.steps, MIN_TIMED_MS, dev, D.barrier, "step")
     wall = time.perf_counter() - wall0
     clocks = sampler.stop()
-    gemm_status = max(wush.linear_status(d_["ws"], M, K, g) for d_ in sets)
+    gemm_status = wl.status()
 
     # ---- per-kernel durations: the same launches, one kind per graph
-    q_ms, _ = timed(quant_only, args.steps, "quantiser")
-    g_ms, _ = timed(gemm_only, args.steps, "gemm")
+    q_ms, q_rep, _, _ = timed(wl.quant_only, sets, args.steps, MIN_TIMED_MS_SIDE, dev, None, "quantiser")
+    g_ms, g_rep, _, _ = timed(wl.gemm_only, sets, args.steps, MIN_TIMED_MS_SIDE, dev, None, "gemm")
 
     # ---- cuBLAS bf16 GEMM of the same shape (the paper's normaliser), same protocol
+    W = wl.W
     Wb = [W] + [W.clone() for _ in range(max(1, min(3, int(252e6 // (W.numel() * 2)))))]
     Yb = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
     nb = len(Wb)
@@ -272,7 +381,9 @@ def run_ours(args):
         _c[0] += 1
         torch.matmul(d_["X"], Wb[_c[0] % nb].t(), out=Yb)
 
-    bf16_ms, _ = timed(bf16_step, args.steps, "bf16 gemm")
+    bf16_ms, _, _, _ = timed(bf16_step, sets, args.steps, MIN_TIMED_MS_SIDE, dev, None, "bf16 gemm")
+    del Wb, Yb
+    lib_ms = library_fp4_gemm_ms(wl, args.steps, dev) if rank == 0 else None
 
     # ---- the two offline kernels of the path (Algorithm 2), timed once each for the record
     def once(fn, reps=5):
@@ -284,6 +395,7 @@ def run_ours(args):
         b_.record(stream)
         torch.cuda.synchronize()
         return a_.elapsed_time(b_) / reps
+    layer = wl.layer
     # moments of the weight matrix itself (the larger of the two inputs of Algorithm 2), caller-owned buffers
     mom_buf = torch.zeros((K // g, g, g), dtype=torch.float32, device=dev)
     cnt_buf = torch.zeros(2, dtype=torch.int64, device=dev)
@@ -293,12 +405,13 @@ def run_ours(args):
               torch.zeros(4, dtype=torch.float32, device=dev), torch.empty(256, dtype=torch.uint8, device=dev))
     wq_ms = once(lambda: wush.quantize_weight(W, layer.Tinv, fmt, sf=wush.SF_TILED, out=wq_out), reps=10)
     offline = {"calib_moments": {"ms": mom_ms, "GB/s": (2.0 * N * K + 4.0 * K * g) / (mom_ms * 1e-3) / 1e9, "rows": N,
-                                 "note": "second-moment sums of W[N,K]; warm L2 (same buffers every repetition)"},
+                                 "note": "second-moment sums of W[N,K]; same buffers every repetition"},
                "quantize_weight": {"ms": wq_ms, "GB/s": (2.0 * N * K * (2 if fmt == "nvfp4" else 1) + N * K / 2.0 + N * K / g) / (wq_ms * 1e-3) / 1e9,
-                                   "note": "NVFP4 reads W twice (AbsMax pass + quantise pass); warm L2"}}
+                                   "note": "NVFP4 reads W twice (AbsMax pass + quantise pass)"}}
+    del wq_out, mom_ws
 
     # ---- end to end through the public call with HOST buffers: pinned X in, Y back out, every step
-    Xh = torch.from_numpy(Xh_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Xh = torch.from_numpy(wl.Xh_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
     n_e2e = max(6, min(args.steps, 60))
     # Three streams: the pinned-host -> device copy of step i+1, the kernels of step i and the device -> host
     # copy of step i-1 overlap (the copy engines are full duplex); every step still moves its own input in
@@ -308,7 +421,7 @@ def run_ours(args):
     ev_in = [torch.cuda.Event() for _ in range(nb3)]
     ev_c = [torch.cuda.Event() for _ in range(nb3)]
     ev_out = [torch.cuda.Event() for _ in range(nb3)]
-    Yh3 = [torch.empty((M, N), dtype=out_dtype).pin_memory() for _ in range(nb3)]
+    Yh3 = [torch.empty((M, N), dtype=wl.out_dtype).pin_memory() for _ in range(nb3)]
 
     def e2e_loop(n):
         for i in range(n):
@@ -321,7 +434,7 @@ def run_ours(args):
             with torch.cuda.stream(s_c):
                 s_c.wait_event(ev_in[b])
                 s_c.wait_event(ev_out[b])                # the previous result in this Y buffer has left
-                step(d_)
+                wl.step(d_)
                 ev_c[b].record(s_c)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_c[b])
@@ -330,6 +443,7 @@ def run_ours(args):
 
     e2e_loop(3)
     torch.cuda.synchronize()
+    gemm_status = max(gemm_status, wl.status())
     D.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -341,9 +455,11 @@ def run_ours(args):
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms_rank = e0.elapsed_time(e1) / n_e2e
-    X, Y = sets[0]["X"], sets[0]["Y"]
+    h2d_bytes = int(sets[0]["X"].numel() * 2)
+    d2h_bytes = int(sets[0]["Y"].numel() * sets[0]["Y"].element_size())
+    del Yh3, Xh, sets, layer, mom_buf, cnt_buf
 
-    flops = 2.0 * M * N * K
+    flops = wl.flops
     rate, t_max = D.whole_job_rate(flops, ms_rank * 1e-3, dev)
     e2e_rate, _ = D.whole_job_rate(flops, e2e_ms_rank * 1e-3, dev)
     D.barrier()
@@ -364,111 +480,107 @@ def run_ours(args):
         traffic = {}
     fp4_peak = peaks["bf16_tflops"] * 4.0
     gemm_tf = flops / (g_ms * 1e-3) / 1e12
-    q_bytes = 2.0 * M * K + M * K / 2.0 + M * K / g + 2.0 * K * g
+    q_bytes = wl.q_bytes
     q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
-    # DRAM bytes per launch from the ncu capture of the same kernel and workload (none for other token counts,
-    # except M <= 128 on config 5, where the weights are the traffic whatever M is)
+    # DRAM bytes per launch from the ncu capture of the same kernel, keyed by workload and token count
     gemm_kernel = "gemm_fp4_2cta_kernel" if M > 128 else "gemm_fp4_kernel"
-    same_workload = (M == cfg.M) or (M <= 128 and cfg.index == 5)
-    gemm_traffic = traffic.get(f"{gemm_kernel}/config{cfg.index}") if same_workload else None
-    roof = {"bound": "tensor", "kernel": "gemm_fp4_2cta_kernel" if M > 128 else "gemm_fp4_kernel", "achieved": gemm_tf, "peak": fp4_peak, "unit": "TFLOP/s",
-            "frac": gemm_tf / fp4_peak, "traffic": gemm_traffic, "ms": g_ms,
+    tkey = f"config{cfg.index}" + (f"_m{M}" if cfg.m_sweep and M > 128 else "")
+    gemm_traffic = traffic.get(f"{gemm_kernel}/{tkey}")
+    roof = {"bound": "tensor", "kernel": gemm_kernel, "achieved": gemm_tf, "peak": fp4_peak, "unit": "TFLOP/s",
+            "frac": gemm_tf / fp4_peak, "traffic": gemm_traffic, "ms": g_ms, "replays": g_rep,
             "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TF/s x 4 (nominal FP4:bf16)",
-            "frac_of_spec_9pf": gemm_tf / 9000.0,
-            # the timed graph replays the kernel back to back for milliseconds, i.e. under the power cap: the
-            # sustained bf16 figure x 4 is the like-for-like ceiling; "frac" keeps the stricter burst figure
+            "frac_of_spec_9pf": gemm_tf / FP4_SPEC_TFLOPS,
+            # the timed graphs replay the kernel back to back for tens of milliseconds, i.e. under the power cap:
+            # the sustained bf16 figure x 4 is the like-for-like ceiling; "frac" keeps the stricter burst figure
             "peak_sustained": peaks["bf16_tflops_sustained"] * 4.0,
             "frac_of_sustained": gemm_tf / (peaks["bf16_tflops_sustained"] * 4.0)}
     if M <= 128:
         # decode regime: the GEMM reads every weight byte once and does almost no arithmetic per byte, so its
         # roofline is HBM: algorithmic bytes (codes + scales of X~ and W~, plus Y) over the measured copy rate
-        g_bytes = M * K / 2.0 + M * K / g + N * K / 2.0 + N * K / g + M * N * (2 if args.out == "bf16" else 4)
-        g_gbs = g_bytes / (g_ms * 1e-3) / 1e9
+        g_gbs = wl.g_bytes / (g_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": gemm_kernel, "achieved": g_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": g_gbs / peaks["hbm_gbs"], "traffic": gemm_traffic, "ms": g_ms, "algorithmic_bytes": g_bytes,
-                "peak_source": peaks["source"], "frac_of_spec_8tbs": g_gbs / 8000.0, "tflops": gemm_tf}
+                "frac": g_gbs / peaks["hbm_gbs"], "traffic": gemm_traffic, "ms": g_ms, "replays": g_rep,
+                "algorithmic_bytes": wl.g_bytes, "peak_source": peaks["source"], "frac_of_spec_8tbs": g_gbs / HBM_SPEC_GBS,
+                "tflops": gemm_tf}
     roof_q = {"bound": "hbm", "kernel": "tq_stream_kernel", "achieved": q_gbs, "peak": peaks["hbm_gbs"],
-              "unit": "GB/s", "frac": q_gbs / peaks["hbm_gbs"], "traffic": traffic.get(f"tq_stream_kernel/config{cfg.index}") if M == cfg.M else None, "ms": q_ms,
-              "algorithmic_bytes": q_bytes, "peak_source": peaks["source"], "frac_of_spec_8tbs": q_gbs / 8000.0}
+              "unit": "GB/s", "frac": q_gbs / peaks["hbm_gbs"], "traffic": traffic.get(f"tq_stream_kernel/{tkey}"), "ms": q_ms,
+              "replays": q_rep, "algorithmic_bytes": q_bytes, "peak_source": peaks["source"], "frac_of_spec_8tbs": q_gbs / HBM_SPEC_GBS}
+    set_mb = wl.set_bytes / 1e6
+
+    # ---- the other benchmark shapes, same protocol (single-GPU runs only; shares W and calibration of config 5)
+    others = []
+    if world == 1 and not args.no_workloads:
+        shared = (wl.W, wl.Xc) if cfg.index == 5 else (None, None)
+        wl.release()
+        plan = [(5, "mxfp4", 4096), (5, "nvfp4", 4096), (5, "mxfp4", 128), (5, "mxfp4", 1), (3, "mxfp4", None),
+                (4, "mxfp4", None), (4, "nvfp4", None), (2, "nvfp4", None)]
+        cache = {5: shared}
+        for ci, f_, m_ in plan:
+            c_ = synth.CONFIGS[ci]
+            m_ = c_.M if m_ is None else m_
+            if (ci, f_, m_) == (cfg.index, fmt, M):
+                continue
+            try:
+                Wd, Xcd = cache.get(ci, (None, None))
+                w2 = Workload(c_, f_, m_, dev, args.out, "wush", False, W=Wd, Xc=Xcd)
+                cache = {ci: (w2.W, w2.Xc)}               # keep one shape's inputs on the device at a time
+                for i in range(3):
+                    w2.step(w2.sets[i % w2.nsets])
+                torch.cuda.synchronize()
+                k2 = max(4, min(args.steps, 50))
+                s_ms, _, _, _ = timed(w2.step, w2.sets, k2, MIN_TIMED_MS_SIDE, dev, None, "step")
+                qq, _, _, _ = timed(w2.quant_only, w2.sets, k2, MIN_TIMED_MS_SIDE, dev, None, "quantiser")
+                gg, _, _, _ = timed(w2.gemm_only, w2.sets, k2, MIN_TIMED_MS_SIDE, dev, None, "gemm")
+                e = {"workload": c_.name, "M": m_, "K": c_.K, "N": c_.N, "format": f_, "status": w2.status()}
+                e.update(fractions(w2, peaks, s_ms, qq, gg))
+                others.append(e)
+                w2.release()
+                del w2
+            except Exception as exc:       # pragma: no cover
+                others.append({"workload": c_.name, "M": m_, "format": f_, "error": str(exc)[:200]})
+        cache = None
+    else:
+        wl.release()
 
     cpu = None
     if not args.no_cpu_baseline:
         rows = min(M, args.ref_rows)
-        sec, passes = oracle_sample_seconds(cfg, fmt, M, rows, dynamic)
+        sec, passes = oracle_sample_seconds(cfg, fmt, M, rows, wl.dynamic)
         cpu = {"value": 2.0 * rows * N * K / sec / 1e12, "unit": "TFLOP/s", "cores": host_threads(), "kind": "oracle",
                "sample": f"{rows} of {M} token rows x all N per pass of the online path (fp64 numpy); "
                          f"{passes} passes, {sec:.2f} s each, {sec * passes:.0f} s of CPU work"}
 
     line = {"metric": METRIC, "value": rate / 1e12, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": t_max * 1e3, "higher_is_better": True, "scaling": "weak",
+            "warmup": warm, "ms_per_step": t_max * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4_e2m1 (fp32 accumulate)", "data": "synthetic",
-            "config": {"workload": cfg.name, "M": M, "K": K, "N": N, "format": fmt, "g": g, "y_dtype": args.out, "transform": args.transform,
-                       "x_tensor_scale": ("per batch" if dynamic else "static") if fmt == "nvfp4" else None,
-                       "l2": f"cold data: {nsets} rotating buffer sets of {set_bytes / 1e6:.0f} MB (> 2x L2)",
-                       "launch": "one CUDA graph of K steps" if used_graph else "eager loop", "tokens_per_rank": M},
+            "replays": replays, "ms_per_step_min": min(per_replay), "ms_per_step_max": max(per_replay),
+            "config": config_of(args, cfg, fmt, M),
+            "timing": {"l2": f"cold data: {nsets} rotating buffer sets of {set_mb:.0f} MB (> 2x L2)",
+                       "launch": (f"one CUDA graph of K steps, replayed {replays} times ({replays * args.steps * ms_rank:.0f} ms timed); "
+                                  "median replay") if used_graph else "eager loop"},
             "roofline": roof, "roofline_quant": roof_q,
             "bf16_gemm": {"ms": bf16_ms, "tflops": flops / (bf16_ms * 1e-3) / 1e12, "speedup_linear": bf16_ms / ms_rank,
                           "speedup_gemm_only": bf16_ms / g_ms, "impl": "torch.matmul (cuBLAS)"},
-            "e2e": {"value": e2e_rate / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": int(X.numel() * 2),
-                    "d2h_bytes_per_step": int(Y.numel() * Y.element_size()), "ms_per_step": e2e_ms_rank},
-            "gpu_launches": (3 if dynamic else 2) * args.steps, "kernel_ms": {"transform_quant": q_ms, "gemm_fp4": g_ms},
-            "gemm_status": gemm_status, "offline_kernels": offline, "clocks": clocks, "wall_s_timed_region": wall, "cpu_baseline": cpu}
+            "fp4_gemm_library": None if lib_ms is None else
+            {"ms": lib_ms, "tflops": flops / (lib_ms * 1e-3) / 1e12, "ours_over_library": lib_ms / g_ms,
+             "impl": "torch._scaled_mm (cuBLASLt block-scaled FP4), context only"},
+            "e2e": {"value": e2e_rate / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d_bytes,
+                    "d2h_bytes_per_step": d2h_bytes, "ms_per_step": e2e_ms_rank},
+            "gpu_launches": (3 if wl.dynamic else 2) * args.steps, "kernel_ms": {"transform_quant": q_ms, "gemm_fp4": g_ms},
+            "gemm_status": gemm_status, "offline_kernels": offline, "clocks": clocks, "wall_s_timed_region": wall,
+            "workloads": others, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     D.shutdown()
-
-
-def run_quantiser_sweep(args):
-    """`--quantiser-sweep`: wush_quantize_act alone over seven activation shapes, both formats, on a GPU that
-    runs nothing else (0.3 s idle before every timed replay), one line of JSON per shape.  Random bf16 data
-    and transforms: the kernel's time does not depend on the values."""
-    import torch
-    from paper_2512_00956_b200 import wush
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
-    reps = 20
-    for M, K in ((2048, 4096), (1024, 8192), (4096, 4096), (4096, 8192), (4096, 14336), (8192, 8192), (16384, 8192)):
-        for fmt, g in (("mxfp4", 32), ("nvfp4", 16)):
-            nset = max(2, int(300e6 // (M * K * 2)) + 1)            # cold data: more than twice the L2 between reuses
-            Xs = [torch.randn(M, K, device=dev).to(torch.bfloat16) for _ in range(nset)]
-            T = (torch.randn(K // g, g, g, device=dev) / g ** 0.5).to(torch.bfloat16)
-            outs = [(torch.empty(M, K // 2, dtype=torch.uint8, device=dev),
-                     torch.zeros(wush.scale_bytes(M, K, g, wush.SF_TILED), dtype=torch.uint8, device=dev)) for _ in range(nset)]
-            ts = torch.tensor([0.01], device=dev) if fmt == "nvfp4" else None
-            side = torch.cuda.Stream(device=dev)
-            with torch.cuda.stream(side):
-                for i in range(3):
-                    wush.quantize_act(Xs[i % nset], T, fmt, ts, wush.SF_TILED, out=outs[i % nset])
-                side.synchronize()
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(graph, stream=side):
-                    for i in range(reps):
-                        wush.quantize_act(Xs[i % nset], T, fmt, ts, wush.SF_TILED, out=outs[i % nset])
-                graph.replay()
-                side.synchronize()
-                times = []
-                for _ in range(5):
-                    time.sleep(0.3)
-                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    a.record(side)
-                    graph.replay()
-                    b.record(side)
-                    side.synchronize()
-                    times.append(a.elapsed_time(b) / reps * 1e3)
-            us = statistics.median(times)
-            nbytes = 2.0 * M * K + M * K / 2.0 + M * K / g + 2.0 * K * g
-            print(json.dumps({"kernel": "tq_stream_kernel", "M": M, "K": K, "format": fmt, "us": round(us, 2),
-                              "us_min": round(min(times), 2), "GB/s": round(nbytes / us / 1e3),
-                              "items_per_sm": round((M / 128) * (K / 128) / 148, 1)}), flush=True)
-            del Xs, outs, graph
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="workload index 1..5 (2 = the headline configuration)")
+    ap.add_argument("--config", type=int, default=5,
+                    help="workload index 1..5 (default 5: the largest single-GPU one, at its largest token count)")
     ap.add_argument("--fmt", default=None, choices=[None, "mxfp4", "nvfp4", "mxfp4_ceil"])
     ap.add_argument("--dynamic-ts", action="store_true",
                     help="NVFP4: activation tensor scale from each batch (one more kernel per step) instead of calibration")
@@ -479,12 +591,8 @@ def main():
                          "one shared Hadamard, or none")
     ap.add_argument("--ref-rows", type=int, default=1024, help="token rows in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--quantiser-sweep", action="store_true",
-                    help="time wush_quantize_act alone over seven shapes (one JSON line each) and exit")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the `workloads` array (the other shapes)")
     args = ap.parse_args()
-    if args.quantiser_sweep:
-        run_quantiser_sweep(args)
-        return
     if args.impl == "reference":
         run_reference(args)
     else:

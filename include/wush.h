@@ -107,7 +107,11 @@ size_t wush_scale_bytes(int64_t rows, int64_t K, int g, wush_sf_layout_t sf);
  *   x_tensor_scale  fp32[1] on the device; NVFP4 only (static, chosen at calibration
  *          time), must be > 0; pass NULL for MXFP4.
  *   codes  uint8 [M, K/2];  scales uint8, layout `sf`.
- * Errors: NULL / SHAPE / FORMAT / ALIGN / CUDA.  M = 0 is a no-op returning WUSH_OK. */
+ * Errors: NULL / SHAPE / FORMAT / ALIGN / CUDA.  M = 0 is a no-op returning WUSH_OK.
+ * Stand-alone, this call has no status word (wush_linear has): its waits are bounded like all others, but an
+ * expired one goes unreported and leaves part of the outputs unwritten.
+ * For NVFP4 the tensor scale is read on the device when the kernel runs, so it may be the output of work
+ * enqueued earlier on the same stream (wush_act_tensor_scale directly before this call, for example). */
 int wush_quantize_act(const void* X, int64_t M, int64_t K, const void* T,
                       wush_format_t fmt, int g, const float* x_tensor_scale,
                       uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf, void* stream);
@@ -173,14 +177,24 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T,
                 void* workspace, size_t workspace_bytes, void* stream);
 size_t wush_linear_workspace_bytes(int64_t M, int64_t K, int g);
 
+/* One size for a workspace that serves every call of a layer with d_batch <= M tokens, d_out = N and d_in = K
+ * (the arguments of the problem statement, Sec. 3 "Problem setup"): the largest of
+ * wush_linear_workspace_bytes(M, K, g), wush_quantize_weight_workspace_bytes(N, K, fmt, g) and
+ * wush_calib_moments_workspace_bytes(max(M, N), K, g) - calibration chunks of up to max(M, N) rows, which
+ * covers the weight matrix itself.  0 on bad arguments. */
+size_t wush_workspace_bytes(int64_t M, int64_t N, int64_t K, wush_format_t fmt, int g);
+
 /* Offline calibration statistics (Algorithm 2, first line of the RTN loop):
  *   moments[c] += sum_t  x_{t,c}^T x_{t,c}   (unnormalised g x g second moment of block c)
  *   *count     += B
  *   Xc       bf16 [B,K] (calibration activations, or the weight matrix W[N,K] itself
  *            for the weight-side moment);  moments fp32 [K/g][g][g], accumulated in
  *            place so calibration can be fed in chunks; count int64[1] on the device.
- *   workspace device scratch of at least wush_calib_moments_workspace_bytes(B,K,g).
- * The reduction order is fixed, so results are run-to-run identical. */
+ *   workspace device scratch of at least wush_calib_moments_workspace_bytes(B,K,g): the per-CTA partial sums
+ *            of the first kernel, added up in a fixed order by the second (no floating-point atomics).
+ * The reduction order is fixed, so results are run-to-run identical.  count must be 8-byte aligned.
+ * This call has no status word: should one of its bounded waits expire, the affected moments are written
+ * as NaN, so a failed call cannot be mistaken for a result. */
 int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* moments,
                        int64_t* count, void* workspace, size_t workspace_bytes, void* stream);
 size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g);
@@ -202,9 +216,19 @@ size_t wush_calib_moments_workspace_bytes(int64_t B, int64_t K, int g);
 int wush_build_transforms(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x,
                           int64_t K, int g, float lambda, void* T, float* Tinv, int32_t* info,
                           void* stream);
-/* The same with a choice of transform: WUSH_KIND_WUSH (the call above) or WUSH_KIND_WUS, the ablation of
- * Sec. 6 / Table 1 "WUSH without Hadamard", T = S^-1/2 U^T W'^T.  Errors as above; FORMAT for another kind. */
-typedef enum { WUSH_KIND_WUSH = 0, WUSH_KIND_WUS = 1 } wush_transform_kind_t;
+/* The same with a choice of transform: WUSH_KIND_WUSH (the call above), WUSH_KIND_WUS, the ablation of
+ * Sec. 6 / Table 1 "WUSH without Hadamard", T = S^-1/2 U^T W'^T, or one of the two fixed transforms described
+ * at the enum.  Errors as above; FORMAT for another kind. */
+typedef enum {
+  WUSH_KIND_WUSH = 0,
+  WUSH_KIND_WUS = 1,
+  /* The two data-independent comparison transforms of Sec. 5 ("H + Quant", "None + Quant") and Table 1: the same
+   * normalised Sylvester-Hadamard matrix H[j][k] = (-1)^popcount(j & k) / sqrt(g) for every block, or the
+   * identity.  mom_w, mom_x, rows_w, rows_x and lambda are ignored (the pointers may be NULL); T receives the
+   * bf16-rounded matrix replicated K/g times, Tinv the inverse-transpose of those stored values. */
+  WUSH_KIND_HADAMARD = 2,
+  WUSH_KIND_IDENTITY = 3
+} wush_transform_kind_t;
 int wush_build_transforms_kind(const float* mom_w, int64_t rows_w, const float* mom_x, int64_t rows_x,
                                int64_t K, int g, float lambda, wush_transform_kind_t kind, void* T,
                                float* Tinv, int32_t* info, void* stream);
@@ -254,12 +278,18 @@ int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, i
  * of x that differ in mismatches[i] (uint64, device array; expected: all zero).  About 1 ms per divisor. */
 int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void* stream);
 /* Test hook for the persistent GEMM (M > 128): use at most `clusters` two-CTA clusters in later calls on the
- * calling thread's current device (0 = as many as fit, the default).  With few clusters even a small problem
+ * current device (0 = as many as fit, the default; the setting is per device, shared by all threads).  With few clusters even a small problem
  * gives every cluster several tiles in a row, which is how the tests reach the hand-over between tiles
  * (accumulator drained while the next tile's loads run) without a full-size input.  Results never depend
  * on it.  Returns the previous value. */
 int wush_debug_gemm_clusters(int clusters);
-/* Test hook for the error path: the next wush_linear call on the calling thread's current device leaves the
+/* Test hook for the streaming quantiser: tile height of later wush_quantize_act / wush_quantize_act_dynamic /
+ * wush_linear calls on the current device (a per-device setting) - 64 or 128 token rows, 0 = chosen from the problem
+ * size (the default: 128 once every SM gets at least five 128 x 128 items).  The tests use it to run ragged token
+ * counts and channel tails through both instantiations without full-size inputs.  Results never depend on it.
+ * Returns the previous value, or WUSH_ERR_SHAPE for another height. */
+int wush_debug_quantiser_rows(int rows);
+/* Test hook for the error path: the next wush_linear call on the current device (whichever thread makes it) leaves the
  * tile of work item `item` of its quantiser kernel unrequested (one call only; -1 cancels).  The consumers'
  * bounded wait for that tile (about a second) then expires, the status word is set, both kernels of the
  * call still complete and the next call works as usual.  Nothing faults and nothing waits without a bound. */

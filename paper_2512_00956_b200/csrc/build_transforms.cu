@@ -267,6 +267,32 @@ cudaError_t run_invert_transforms(const void* T, int64_t K, int g, float* Tinv, 
   return cudaGetLastError();
 }
 
+// The data-independent comparison transforms of Sec. 5 / Table 1 written in the layout the kernels take: the
+// same normalised Sylvester-Hadamard matrix (kind 0; entries +-d^-1/2 rounded to bf16) or the identity (kind 1)
+// for every block.
+template <int D>
+__global__ void __launch_bounds__(BT_THREADS)
+fixed_transforms_kernel(__nv_bfloat16* __restrict__ T, int kind) {
+  const float h = rsqrtf((float)D);                      // exact for D = 16, one rounding for D = 32; bf16 below
+  for (int idx = threadIdx.x; idx < D * D; idx += BT_THREADS) {
+    const int j = idx / D, k = idx % D;
+    float v;
+    if (kind == 0) v = (__popc(j & k) & 1) ? -h : h;
+    else v = (j == k) ? 1.0f : 0.0f;
+    T[(size_t)blockIdx.x * D * D + idx] = __float2bfloat16_rn(v);
+  }
+}
+
+cudaError_t run_fixed_transforms(int kind, int64_t K, int g, void* T, float* Tinv, int32_t* info, cudaStream_t st) {
+  const int C = (int)(K / g);
+  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(T);
+  if (g == 32) fixed_transforms_kernel<32><<<C, BT_THREADS, 0, st>>>(Tb, kind);
+  else fixed_transforms_kernel<16><<<C, BT_THREADS, 0, st>>>(Tb, kind);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return run_invert_transforms(T, K, g, Tinv, info, st);   // Eq. 6 for the stored values
+}
+
 cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* mom_x, int64_t n_x, int64_t K, int g,
                                  double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st, bool with_hadamard) {
   const int wh = with_hadamard ? 1 : 0;
@@ -275,11 +301,13 @@ cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* m
   __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(T);
   cudaError_t e;
   if (g == 32) {
-    static bool done = false;
-    if (!done) {
+    static bool done_of[kDeviceSlots] = {};              // the attribute belongs to the device's copy of the kernel
+    const int slot = device_slot();
+    if (slot < 0) return cudaErrorInvalidDevice;
+    if (!done_of[slot]) {
       e = cudaFuncSetAttribute(build_transforms_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      done = true;
+      done_of[slot] = true;
     }
     build_transforms_kernel<32><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info, wh);
   } else {

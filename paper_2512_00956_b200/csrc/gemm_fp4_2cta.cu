@@ -21,6 +21,8 @@
 // CTA's own bounded waits expire in turn, so the closing cluster barrier is always reached.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "wush_device.cuh"
 #include "wush_host.h"
 
@@ -257,9 +259,15 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
         __syncwarp();
       }
     }
-    if (!ok) {                                     // give copies already in flight time to land before the CTA exits
+    if (!ok && rank == 0) {
+      // A wait expired.  Copies this pair has already requested must land before either CTA exits: all of them
+      // (both CTAs') count on the leader's full barriers, so the leader waits for the stages requested so far,
+      // with one deadline for all of them, and the peer stays at the closing cluster barrier until the leader
+      // arrives there.  A stage the peer never requested simply runs into the deadline.
       const uint64_t t0 = timer_ns();
-      while (timer_ns() - t0 < 200000ull) { }
+      for (int k = max(0, g - STAGES); k < g; ++k)
+        while (!try_wait(s32(&full_bar[k % STAGES]), (k / STAGES) & 1))
+          if (timer_ns() - t0 > 2000000ull) break;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
@@ -487,13 +495,11 @@ static bool map_output(CUtensorMap* map, void* Y, int64_t M, int64_t N, int out_
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int g_cluster_limit[kDeviceSlots] = {};
+static std::atomic<int> g_cluster_limit[kDeviceSlots];
 int gemm_2cta_cluster_limit(int clusters) {
   const int slot = device_slot();
   if (slot < 0) return 0;
-  const int old = g_cluster_limit[slot];
-  g_cluster_limit[slot] = clusters < 0 ? 0 : clusters;
-  return old;
+  return g_cluster_limit[slot].exchange(clusters < 0 ? 0 : clusters);
 }
 
 template <int FMT>
@@ -527,7 +533,8 @@ static cudaError_t launch_2cta(const CUtensorMap& a, const CUtensorMap& b, const
   }
   const int tiles = ((M + g2::BM - 1) / g2::BM) * ((N + g2::BN - 1) / g2::BN);
   int nc = tiles < clusters ? tiles : clusters;
-  if (g_cluster_limit[slot] > 0 && g_cluster_limit[slot] < nc) nc = g_cluster_limit[slot];
+  const int limit = g_cluster_limit[slot].load();
+  if (limit > 0 && limit < nc) nc = limit;
   if (!pdl) {
     g2::gemm_fp4_2cta_kernel<FMT><<<2 * nc, g2::THREADS, g2::smem_bytes(FMT), st>>>(a, b, sa, sb, M, N, K, tsx, tsw, y,
                                                                                      out_bf16, status, cs);

@@ -161,6 +161,7 @@ extern "C" int wush_calib_moments_static(const void* Xc, int64_t B, int64_t K, i
     return WUSH_ERR_SHAPE;
   if (!Xc || !moments || !count) return WUSH_ERR_NULL;
   if (((reinterpret_cast<uintptr_t>(Xc) | reinterpret_cast<uintptr_t>(moments)) & 15u) != 0) return WUSH_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(count) & 7u) != 0) return WUSH_ERR_ALIGN;
   const size_t per_split = (size_t)K * (size_t)g;                 // floats of one partial set
   if (per_split > wush::kStaticScratchFloats) return WUSH_ERR_WORKSPACE;   // K * g beyond the built-in scratch
   if (B == 0) return WUSH_OK;
@@ -169,7 +170,7 @@ extern "C" int wush_calib_moments_static(const void* Xc, int64_t B, int64_t K, i
   if ((size_t)splits > fit) splits = (int)fit;
   float* scratch = nullptr;
   cudaError_t e = wush::static_scratch(&scratch);
-  if (e == cudaSuccess)
-    e = wush::run_calib_moments(Xc, B, K, g, moments, count, scratch, splits, (cudaStream_t)stream);
-  return e == cudaSuccess ? WUSH_OK : WUSH_ERR_CUDA;
+  if (e != cudaSuccess) return wush::record_cuda_error(e, "address of the built-in scratch array");
+  e = wush::run_calib_moments(Xc, B, K, g, moments, count, scratch, splits, (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : wush::record_cuda_error(e);
 }

@@ -27,15 +27,9 @@
 
 namespace wush {
 
-#ifndef MS_ROWS_CFG
-#define MS_ROWS_CFG 64
-#endif
-constexpr int MS_ROWS = MS_ROWS_CFG;                     // tokens per tile
+constexpr int MS_ROWS = 64;                              // tokens per tile
 constexpr int MS_TQ = MS_ROWS / 32;                      // 32-token parts of a tile, one consumer warp each
-#ifndef MS_CONSUMERS_CFG
-#define MS_CONSUMERS_CFG 8
-#endif
-constexpr int MS_CONSUMERS = MS_CONSUMERS_CFG;
+constexpr int MS_CONSUMERS = 8;
 constexpr int MS_CTAS_PER_SM = 16 / MS_CONSUMERS;        // 16 consumer warps per SM either way
 constexpr int MS_PANEL_SB = MS_CONSUMERS / MS_TQ;        // 32-channel super-blocks per tile (panel)
 constexpr int MS_BOXES = MS_PANEL_SB / 2;                // 64-channel TMA boxes per tile

@@ -114,10 +114,6 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restric
   const bool nv_quant = (FMT == kFmtNV) && !AMAX;
   const bool nv_dynamic = nv_quant && amax_in != nullptr;
   float ts = 1.0f;
-  if (nv_quant && !nv_dynamic) {              // static scale: a calibration constant, not the previous kernel's output
-    ts = *ts_ptr;
-    if (threadIdx.x < 128) nv_mult[threadIdx.x] = nv_mult_of_byte(threadIdx.x, ts);
-  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 32) prefetch_tensormap(&mapX);
   if (threadIdx.x == 0) {
@@ -135,10 +131,13 @@ tq_stream_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restric
   // the status word is only ever set after a bounded wait of about a second has expired, so clearing it
   // here cannot race with a report; it saves wush_linear a separate memset between kernels
   if (clear_status && blockIdx.x == 0 && threadIdx.x == 0 && status != nullptr) *status = 0;
-  if (nv_dynamic) {                           // per-batch tensor scale from the AbsMax pass that ran before
-    ts = nv_tensor_scale(__uint_as_float(*amax_in));
+  if (nv_quant) {
+    // The tensor scale is read only here, after the dependency wait: the static one may have been written by
+    // the kernel just before this one on the stream (wush_act_tensor_scale followed by the first layer call),
+    // the per-batch one always is (the AbsMax pass).
+    ts = nv_dynamic ? nv_tensor_scale(__uint_as_float(*amax_in)) : *ts_ptr;
     if (threadIdx.x < 128) nv_mult[threadIdx.x] = nv_mult_of_byte(threadIdx.x, ts);
-    if (blockIdx.x == 0 && threadIdx.x == 0 && ts_out != nullptr) *ts_out = ts;
+    if (nv_dynamic && blockIdx.x == 0 && threadIdx.x == 0 && ts_out != nullptr) *ts_out = ts;
     __syncthreads();
   }
   // let a programmatic dependent (the GEMM of wush_linear) be scheduled as SMs free up; it still waits
@@ -531,7 +530,7 @@ static cudaError_t launch_stream(const void* X, int64_t M, int64_t K, const void
   if (opt.amax_out != nullptr) {                 // AbsMax pass only (g = 16)
     if (g != 16) return cudaErrorNotSupported;
     tq_stream_kernel<16, true, ROWS, NSPLIT><<<grid, SQ_THREADS, SQ_SMEM, st>>>(map, Tb, M, K, nullptr, nullptr, nullptr, sf, num_rb, n_items,
-                                                                        nullptr, 0, nullptr, reinterpret_cast<float*>(opt.amax_out), 0, -1);
+                                                                        status, cs, nullptr, reinterpret_cast<float*>(opt.amax_out), 0, -1);
     return cudaGetLastError();
   }
   if (!pdl) {
@@ -596,7 +595,8 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   // 128-row tiles unless the problem is small: with fewer than SQ_SMALL of them per CTA the 64-row tiles'
   // finer items win (the first tile lands sooner and the CTAs finish closer together)
   const int64_t items128 = ((K / 32 + 3) / 4) * ((M + 127) / 128);
-  if (items128 < (int64_t)SQ_SMALL * sm_count)
+  const bool rows64 = opt.force_rows ? (opt.force_rows == 64) : (items128 < (int64_t)SQ_SMALL * sm_count);
+  if (rows64)
     return launch_stream<64>(X, M, K, T, g, ts, codes, scales, sf, status, clear_status, pdl, st, opt, sm_count);
   return launch_stream<128>(X, M, K, T, g, ts, codes, scales, sf, status, clear_status, pdl, st, opt, sm_count);
 }

@@ -3,18 +3,24 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "../../include/wush.h"
 #include "wush_device.cuh"
 #include "wush_host.h"
 
 namespace {
-
 thread_local char g_cuda_error[256] = "";
+}
 
-int cuda_fail(cudaError_t e, const char* why = nullptr) {
+int wush::record_cuda_error(cudaError_t e, const char* why) {
   snprintf(g_cuda_error, sizeof(g_cuda_error), "%s%s%s", cudaGetErrorString(e), why ? ": " : "", why ? why : "");
   return WUSH_ERR_CUDA;
 }
+
+namespace {
+
+inline int cuda_fail(cudaError_t e, const char* why = nullptr) { return wush::record_cuda_error(e, why); }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int check_fmt(int fmt, int g) {
   if (fmt == WUSH_MXFP4 || fmt == WUSH_MXFP4_CEIL) return g == 32 ? WUSH_OK : WUSH_ERR_FORMAT;
@@ -30,22 +36,28 @@ inline int check_shape(int64_t rows, int64_t K, int g) {
 inline size_t round16(size_t x) { return (x + 15) & ~size_t(15); }
 // the GEMM knows two formats; the scale rule only matters to the quantisers
 inline int gemm_fmt(int fmt) { return fmt == WUSH_NVFP4 ? wush::kFmtNV : wush::kFmtMX; }
+
+// test hook (wush_debug_drop_tile): work item + 1 that the next streaming-quantiser launch of wush_linear on this
+// device will not load (0 = none); one shot, taken with an atomic exchange so that concurrent callers cannot
+// both consume it
+std::atomic<int> g_drop_item[wush::kDeviceSlots];
+int take_drop_item() {
+  const int slot = wush::device_slot();
+  if (slot < 0) return -1;
+  return g_drop_item[slot].exchange(0) - 1;
+}
+// test hook (wush_debug_quantiser_rows): forced tile height of the streaming quantiser on this device (0 = automatic)
+std::atomic<int> g_force_rows[wush::kDeviceSlots];
+int forced_rows() {
+  const int slot = wush::device_slot();
+  return slot < 0 ? 0 : g_force_rows[slot].load();
+}
+
 inline wush::QuantOpts opts_of(int fmt) {
   wush::QuantOpts o;
   o.mx_ceil = (fmt == WUSH_MXFP4_CEIL);
+  o.force_rows = forced_rows();
   return o;
-}
-
-// test hook (wush_debug_drop_tile): work item the next streaming-quantiser launch of wush_linear on this device
-// will not load; one shot
-int g_drop_item[wush::kDeviceSlots];
-bool g_drop_init = false;
-int take_drop_item() {
-  const int slot = wush::device_slot();
-  if (slot < 0 || !g_drop_init) return -1;
-  const int v = g_drop_item[slot];
-  g_drop_item[slot] = -1;
-  return v;
 }
 
 bool device_is_sm100() {
@@ -115,9 +127,9 @@ int wush_quantize_act_dynamic(const void* X, int64_t M, int64_t K, const void* T
   if ((reinterpret_cast<uintptr_t>(x_tensor_scale) & 7u) != 0) return WUSH_ERR_ALIGN;
   if (M == 0) return WUSH_OK;
   uint32_t* amax = reinterpret_cast<uint32_t*>(x_tensor_scale + 1);
-  cudaError_t e = wush::run_act_amax(X, M, K, T, amax, (cudaStream_t)stream);
+  cudaError_t e = wush::run_act_amax(X, M, K, T, amax, (cudaStream_t)stream, nullptr, false, forced_rows());
   if (e != cudaSuccess) return cuda_fail(e);
-  wush::QuantOpts o;
+  wush::QuantOpts o = opts_of(WUSH_NVFP4);
   o.amax_in = amax;
   o.ts_out = x_tensor_scale;
   e = wush::run_quantize_act(X, M, K, T, g, nullptr, codes, scales, (int)sf, nullptr, false, false, (cudaStream_t)stream, o);
@@ -180,6 +192,16 @@ size_t wush_linear_workspace_bytes(int64_t M, int64_t K, int g) {
   return round16((size_t)(M * (K / 2))) + round16(wush_scale_bytes(M, K, g, WUSH_SF_TILED)) + 16 + 16;
 }
 
+size_t wush_workspace_bytes(int64_t M, int64_t N, int64_t K, wush_format_t fmt, int g) {
+  if (check_fmt(fmt, g) != WUSH_OK || M < 0 || N < 0 || K <= 0 || K % g != 0) return 0;
+  size_t need = wush_linear_workspace_bytes(M, K, g);
+  const size_t wq = wush_quantize_weight_workspace_bytes(N, K, fmt, g);
+  const size_t mom = wush_calib_moments_workspace_bytes(M > N ? M : N, K, g);
+  if (wq > need) need = wq;
+  if (mom > need) need = mom;
+  return need;
+}
+
 int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_t* Wcodes,
                 const uint8_t* Wscales, int64_t N, const float* x_tensor_scale, const float* w_tensor_scale,
                 wush_format_t fmt, int g, void* Y, wush_out_t ydt, void* workspace, size_t workspace_bytes,
@@ -210,12 +232,13 @@ int wush_linear(const void* X, int64_t M, int64_t K, const void* T, const uint8_
   cudaError_t e;
   if (dynamic) {                                  // per-batch tensor scale: AbsMax pass first
     uint32_t* amax = reinterpret_cast<uint32_t*>(ts_dyn + 1);
-    if ((e = wush::run_act_amax(X, M, K, T, amax, (cudaStream_t)stream)) != cudaSuccess) return cuda_fail(e);
+    // the AbsMax pass clears the status word and reports into it; the quantising pass must then leave it alone
+    if ((e = wush::run_act_amax(X, M, K, T, amax, (cudaStream_t)stream, status, true, o.force_rows)) != cudaSuccess) return cuda_fail(e);
     o.amax_in = amax;
     o.ts_out = ts_dyn;
     x_tensor_scale = ts_dyn;                      // what the GEMM multiplies by
   }
-  e = wush::run_quantize_act(X, M, K, T, g, dynamic ? nullptr : x_tensor_scale, xq, xs, WUSH_SF_TILED, status, true, true,
+  e = wush::run_quantize_act(X, M, K, T, g, dynamic ? nullptr : x_tensor_scale, xq, xs, WUSH_SF_TILED, status, !dynamic, true,
                              (cudaStream_t)stream, o);
   if (e != cudaSuccess) return cuda_fail(e);
   const char* why = nullptr;
@@ -237,6 +260,7 @@ int wush_calib_moments(const void* Xc, int64_t B, int64_t K, int g, float* momen
   if (!Xc || !moments || !count) return WUSH_ERR_NULL;
   if (!workspace || workspace_bytes < wush_calib_moments_workspace_bytes(B, K, g)) return WUSH_ERR_WORKSPACE;
   if (!aligned16(Xc) || !aligned16(moments) || !aligned16(workspace)) return WUSH_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(count) & 7u) != 0) return WUSH_ERR_ALIGN;
   if (B == 0) return WUSH_OK;
   cudaError_t e = wush::run_calib_moments(Xc, B, K, g, moments, count, reinterpret_cast<float*>(workspace),
                                           wush::moments_splits(B, K), (cudaStream_t)stream);
@@ -247,6 +271,13 @@ int wush_build_transforms_kind(const float* mom_w, int64_t rows_w, const float* 
                                int g, float lambda, wush_transform_kind_t kind, void* T, float* Tinv, int32_t* info,
                                void* stream) {
   if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
+  if (kind == WUSH_KIND_HADAMARD || kind == WUSH_KIND_IDENTITY) {       // data-independent: the moments are not read
+    if (K <= 0 || K % g != 0) return WUSH_ERR_SHAPE;
+    if (!T || !Tinv) return WUSH_ERR_NULL;
+    if (!aligned16(T) || !aligned16(Tinv)) return WUSH_ERR_ALIGN;
+    const cudaError_t ef = wush::run_fixed_transforms(kind == WUSH_KIND_HADAMARD ? 0 : 1, K, g, T, Tinv, info, (cudaStream_t)stream);
+    return ef == cudaSuccess ? WUSH_OK : cuda_fail(ef);
+  }
   if (kind != WUSH_KIND_WUSH && kind != WUSH_KIND_WUS) return WUSH_ERR_FORMAT;
   if (K <= 0 || K % g != 0 || rows_w <= 0 || rows_x <= 0 || !(lambda >= 0.0f)) return WUSH_ERR_SHAPE;
   if (!mom_w || !mom_x || !T || !Tinv) return WUSH_ERR_NULL;
@@ -289,12 +320,15 @@ int wush_debug_gemm_clusters(int clusters) { return wush::gemm_2cta_cluster_limi
 int wush_debug_drop_tile(int item) {
   const int slot = wush::device_slot();
   if (slot < 0) return WUSH_ERR_CUDA;
-  if (!g_drop_init) {
-    for (int i = 0; i < wush::kDeviceSlots; ++i) g_drop_item[i] = -1;
-    g_drop_init = true;
-  }
-  g_drop_item[slot] = item < 0 ? -1 : item;
+  g_drop_item[slot].store(item < 0 ? 0 : item + 1);
   return WUSH_OK;
+}
+
+int wush_debug_quantiser_rows(int rows) {
+  const int slot = wush::device_slot();
+  if (slot < 0) return WUSH_ERR_CUDA;
+  if (rows != 0 && rows != 64 && rows != 128) return WUSH_ERR_SHAPE;
+  return g_force_rows[slot].exchange(rows);
 }
 
 int wush_decode_status(int32_t word) { return word == 0 ? WUSH_OK : WUSH_ERR_TIMEOUT; }

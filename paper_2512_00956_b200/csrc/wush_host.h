@@ -24,12 +24,17 @@ struct QuantOpts {
   float* ts_out = nullptr;
   uint32_t* amax_out = nullptr;   // run_quantize_act_stream only: AbsMax pass instead of quantising (g = 16)
   int drop_item = -1;             // test hook: the producer never requests this work item (streaming kernel only)
+  int force_rows = 0;             // test hook: 64 or 128 = tile height of the streaming kernel whatever the problem size
 };
+// Text of the last CUDA error of the calling thread (wush_last_cuda_error); returns WUSH_ERR_CUDA.
+int record_cuda_error(cudaError_t e, const char* why = nullptr);
 // clear_status: the kernel zeroes *status itself (wush_linear); otherwise the word is left alone
 cudaError_t run_quantize_act(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                              uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
                              bool pdl, cudaStream_t st, const QuantOpts& opt = QuantOpts());
-cudaError_t run_act_amax(const void* X, int64_t M, int64_t K, const void* T, uint32_t* amax, cudaStream_t st);
+// status / clear_status: as for run_quantize_act (the AbsMax pass reports an expired wait in the same word)
+cudaError_t run_act_amax(const void* X, int64_t M, int64_t K, const void* T, uint32_t* amax, cudaStream_t st,
+                         int32_t* status = nullptr, bool clear_status = false, int force_rows = 0);
 // out[0] = NVFP4 tensor scale of the transformed tokens (AbsMax / 2688, 1 if all zero), out[1] = that AbsMax
 cudaError_t run_act_tensor_scale(const void* X, int64_t M, int64_t K, const void* T, float* out, cudaStream_t st);
 // streaming (TMA-fed, persistent) variant; cudaErrorNotSupported = problem not covered, use the other kernel
@@ -68,6 +73,8 @@ cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* m
                                  double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st,
                                  bool with_hadamard = true);
 cudaError_t run_invert_transforms(const void* T, int64_t K, int g, float* Tinv, int32_t* info, cudaStream_t st);
+// kind 0: one shared normalised Hadamard matrix, kind 1: the identity, for every block; Tinv = T^-T of the stored values
+cudaError_t run_fixed_transforms(int kind, int64_t K, int g, void* T, float* Tinv, int32_t* info, cudaStream_t st);
 
 // two-CTA persistent variant (M > 128); cudaErrorNotSupported = use the single-CTA kernel
 int gemm_2cta_cluster_limit(int clusters);   // test hook: 0 = no limit; returns the previous value (per device)

@@ -4,7 +4,7 @@ Second moments come from the library's calibration kernel (`wush_calib_moments`)
 factorisations of Algorithm 1 and the inverse-transpose of Eq. 6 from `wush_build_transforms`,
 the weight quantisation from `wush_quantize_weight`: nothing leaves the device.  The comparison
 transforms of Sec. 5 / Table 1 (one shared Hadamard matrix, the identity, WUSH without its Hadamard
-factor) go through the same calls; their weight-side partners come from `wush_invert_transforms`.
+factor) come from `wush_build_transforms_kind` as well, so this module holds no arithmetic of its own.
 
 Conventions (the paper leaves them open): damping ratio lambda = 0.01; singular values
 descending and each row of U^T W'^T signed so that its largest-magnitude entry is positive
@@ -12,37 +12,21 @@ descending and each row of U^T W'^T signed so that its largest-magnitude entry i
 transform is stored in bf16 and the weight-side one is the inverse-transpose of the STORED
 values, so that (x T^T)(w Tinv^T)^T = x w^T up to fp32 rounding of Tinv.
 """
-import math
-
 import torch
 
 from . import wush
-
-
-def hadamard(d, device):
-    i = torch.arange(d, device=device)
-    a = i[:, None] & i[None, :]
-    pop = torch.zeros_like(a)
-    for b in range(max(1, d.bit_length())):
-        pop += (a >> b) & 1
-    return torch.where(pop % 2 == 0, 1.0, -1.0).to(torch.float64) / math.sqrt(d)
 
 
 def fixed_transforms(kind, C, d, device):
     """The data-independent comparison transforms of Sec. 5 / Table 1, in the layout the kernels take:
     "hadamard" (the same normalised Hadamard matrix for every block, the H + Quant baseline) or
     "identity" (None + Quant).  Returns (T bf16 [C,d,d], Tinv fp32 [C,d,d]) with Tinv = T^-T of the
-    stored bf16 values, exactly as for WUSH."""
-    if kind == "hadamard":
-        T1 = hadamard(d, device)
-    elif kind == "identity":
-        T1 = torch.eye(d, dtype=torch.float64, device=device)
-    else:
+    stored bf16 values, exactly as for WUSH.  Both are written by the library."""
+    if kind not in ("hadamard", "identity"):
         raise ValueError(kind)
-    T = T1.to(torch.bfloat16).expand(C, d, d).contiguous()
-    Tinv, info = wush.invert_transforms(T, d)                                    # Eq. 6 for the stored values
+    T, Tinv, info = wush.fixed_transforms(kind, C, d, device)
     if int(info.abs().max().item()) != 0:
-        raise wush.WushError("wush_invert_transforms: singular transform")
+        raise wush.WushError("wush_build_transforms_kind: singular transform")
     return T, Tinv
 
 

@@ -27,7 +27,7 @@ EXPORTS = [
     "wush_quantize_f32", "wush_transform_act_f32", "wush_transform_weight_f32", "wush_calib_moments_static",
     "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division", "wush_debug_gemm_clusters",
     "wush_debug_drop_tile", "wush_decode_status", "wush_build_transforms_kind", "wush_invert_transforms",
-    "wush_act_tensor_scale",
+    "wush_act_tensor_scale", "wush_workspace_bytes", "wush_debug_quantiser_rows",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -60,6 +60,10 @@ def lib():
         L.wush_linear.argtypes = [vp, i64, i64, vp, vp, vp, i64, vp, vp, i32, i32, vp, i32, vp, sz, vp]
         L.wush_linear_workspace_bytes.restype = sz
         L.wush_linear_workspace_bytes.argtypes = [i64, i64, i32]
+        L.wush_workspace_bytes.restype = sz
+        L.wush_workspace_bytes.argtypes = [i64, i64, i64, i32, i32]
+        L.wush_debug_quantiser_rows.argtypes = [i32]
+        L.wush_debug_quantiser_rows.restype = i32
         L.wush_calib_moments.argtypes = [vp, i64, i64, i32, vp, vp, vp, sz, vp]
         L.wush_calib_moments_workspace_bytes.restype = sz
         L.wush_calib_moments_workspace_bytes.argtypes = [i64, i64, i32]
@@ -193,6 +197,12 @@ def linear_workspace_bytes(M, K, g):
     return lib().wush_linear_workspace_bytes(M, K, g)
 
 
+def workspace_bytes(M, N, K, fmt):
+    """One workspace size that serves every call of a layer with up to M tokens (wush_workspace_bytes)."""
+    f, g = _fmt(fmt)
+    return lib().wush_workspace_bytes(M, N, K, f, g)
+
+
 def linear(X, T, Wcodes, Wscales, fmt, x_tensor_scale=None, w_tensor_scale=None, out_dtype=torch.float32,
            out=None, workspace=None):
     """The whole online layer: Y = q(X T^T) (x) W~ (Eq. 7).  Returns (Y, workspace).
@@ -239,7 +249,19 @@ def calib_moments(Xc, g, moments=None, count=None, workspace=None):
     return moments, count
 
 
-KINDS = {"wush": 0, "wus": 1}
+KINDS = {"wush": 0, "wus": 1, "hadamard": 2, "identity": 3}
+
+
+def fixed_transforms(kind, C, g, device):
+    """The data-independent transforms "hadamard" / "identity" for C blocks, made by the library
+    (wush_build_transforms_kind without moments).  Returns (T bf16 [C,g,g], Tinv fp32 [C,g,g], info)."""
+    T = torch.empty((C, g, g), dtype=torch.bfloat16, device=device)
+    Tinv = torch.empty((C, g, g), dtype=torch.float32, device=device)
+    info = torch.zeros(max(C, 4), dtype=torch.int32, device=device)
+    with torch.cuda.device(device):
+        check(lib().wush_build_transforms_kind(None, 0, None, 0, C * g, g, 0.0, KINDS[kind], _ptr(T), _ptr(Tinv),
+                                               _ptr(info), _stream()))
+    return T, Tinv, info[:C]
 
 
 def build_transforms(mom_w, rows_w, mom_x, rows_x, g, lam=0.01, kind="wush"):
@@ -297,6 +319,14 @@ def debug_drop_tile(item):
 def decode_status(word):
     """WUSH_OK (0) or WUSH_ERR_TIMEOUT for a status word read back from the device."""
     return int(lib().wush_decode_status(int(word)))
+
+
+def debug_quantiser_rows(rows):
+    """Test hook: tile height (64 / 128, 0 = automatic) of the streaming quantiser; returns the old value."""
+    r = int(lib().wush_debug_quantiser_rows(int(rows)))
+    if r < 0:
+        check(r)
+    return r
 
 
 def debug_gemm_clusters(clusters):

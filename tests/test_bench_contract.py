@@ -25,7 +25,7 @@ def test_reference_arm_prints_one_json_line_with_the_contract_keys():
     assert d["impl"] == "reference" and d["unit"] == "TFLOP/s" and d["higher_is_better"] is True
     assert d["steps"] == 1 and d["warmup"] == 0 and d["n_gpus"] == 1 and d["vs_baseline"] is None
     assert d["dtype"] == "f64" and d["data"] == "synthetic" and d["value"] > 0 and d["ms_per_step"] > 0
-    assert d["config"]["workload"] and d["config"]["sample_rows"] == 16
+    assert d["config"]["workload"] and d["sample_rows"] == 16 and "model" not in d["config"]
     cb = d["cpu_baseline"]
     assert cb["kind"] == "oracle" and cb["cores"] >= 1 and cb["value"] == d["value"] and "sample" in cb
     e2e = d["e2e"]

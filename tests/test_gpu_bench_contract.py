@@ -11,7 +11,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def test_bench_line_on_the_small_configuration():
-    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--config", "1", "--steps", "6", "--warmup", "3", "--ref-rows", "32"]
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--config", "1", "--steps", "6", "--warmup", "3", "--ref-rows", "32", "--no-workloads"]
     res = subprocess.run(cmd, capture_output=True, text=True, cwd=ROOT, timeout=600)
     assert res.returncode == 0, res.stderr[-800:]
     lines = [ln for ln in res.stdout.splitlines() if ln.strip()]
@@ -21,6 +21,8 @@ def test_bench_line_on_the_small_configuration():
     assert d["n_gpus"] == 1 and d["steps"] == 6 and d["warmup"] == 3 and d["data"] == "synthetic"
     assert d["value"] > 0 and d["ms_per_step"] > 0 and d["gemm_status"] == 0
     assert d["gpu_launches"] == 2 * d["steps"]
+    assert d["replays"] >= 3 and d["ms_per_step_min"] <= d["ms_per_step"] <= d["ms_per_step_max"]
+    assert d["clocks"]["samples"] >= 10 and d["workloads"] == []
     assert d["config"]["workload"] and "model" not in d["config"]
     r = d["roofline"]
     assert r["bound"] in ("hbm", "tensor") and r["unit"] in ("GB/s", "TFLOP/s")

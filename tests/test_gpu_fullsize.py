@@ -78,14 +78,16 @@ def test_config5_token_sweep(fmt):
         _check_layer(cfg, fmt, M, W_bits, Xc_bits, seed=M, rows=32, check_codes=(M <= 4096))
 
 
-def test_config5_full_width_sampled_channels():
-    """All 28672 output channels on the GPU (MXFP4); the oracle prepares 512 sampled channels."""
+@pytest.mark.parametrize("fmt,M", [("mxfp4", 4096), ("nvfp4", 4096), ("nvfp4", 16384)])
+def test_config5_full_width_sampled_channels(fmt, M):
+    """All 28672 output channels on the GPU; the oracle prepares 512 sampled channels (and, for NVFP4, the
+    tensor scale of the whole transformed weight matrix, which needs the transform but not the quantiser)."""
     cfg = synth.CONFIGS[5]
-    fmt, g, M = "mxfp4", 32, 4096
+    g = G[fmt]
     W_bits = synth.weights(cfg)
     Xc_bits = synth.calibration(cfg)
     X_bits = synth.activations(cfg, M=M)
-    rng = np.random.default_rng(5)
+    rng = np.random.default_rng(5 + M)
     cols = np.sort(rng.choice(cfg.N, size=512, replace=False))
     rows = np.sort(rng.choice(M, size=64, replace=False))
     # transforms depend on the weight moments of ALL channels: take them from the full matrix
@@ -96,15 +98,26 @@ def test_config5_full_width_sampled_channels():
     from oracle import wush_transform as WT
     T_bits, T_hat, T_xvsh = WT.build_transforms(momW, momX, 0.01)
     Tx32 = np.ascontiguousarray(T_xvsh, dtype=np.float32)
+    ts_w = ts_x = None
+    if fmt == "nvfp4":
+        amax_w = 0.0
+        for r0 in range(0, cfg.N, 4096):          # AbsMax of the whole transformed tensor, in slices
+            amax_w = max(amax_w, float(np.max(np.abs(P.transform_blocks(Wv[r0:r0 + 4096], Tx32.astype(np.float64)).astype(np.float32)))))
+        ts_w = np.float32(np.float32(amax_w) / np.float32(2688.0))
+        ts_x = Q.nvfp4_tensor_scale(P.transform_blocks(Xcv, T_hat).astype(np.float32))
     wbar = P.transform_blocks(Wv[cols], Tx32.astype(np.float64)).astype(np.float32)
-    wc, wsb = Q.quantize(wbar, fmt)
-    wdeq = Q.dequantize(wc, wsb, fmt)
-    v32, xc, xs = P.quantize_transformed(F.bf16_bits_to_f64(X_bits[rows]), T_hat, fmt)
-    Yo = P.dequantized_product(Q.dequantize(xc, xs, fmt), wdeq)
+    del Wv
+    wc, wsb = Q.quantize(wbar, fmt, ts_w)
+    wdeq = Q.dequantize(wc, wsb, fmt, ts_w)
+    v32, xc, xs = P.quantize_transformed(F.bf16_bits_to_f64(X_bits[rows]), T_hat, fmt, ts_x)
+    Yo = P.dequantized_product(Q.dequantize(xc, xs, fmt, ts_x), wdeq)
     X, W = dev_bf16(X_bits), dev_bf16(W_bits)
-    wq, ws, _ = wush.quantize_weight(W, dev(Tx32), fmt, sf=wush.SF_TILED)
-    Y, wsp = wush.linear(X, dev_bf16(T_bits), wq, ws, fmt)
+    wq, ws, tsw_g = wush.quantize_weight(W, dev(Tx32), fmt, sf=wush.SF_TILED)
+    tsx_g = dev(np.full(4, ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
+    Y, wsp = wush.linear(X, dev_bf16(T_bits), wq, ws, fmt, tsx_g, tsw_g)
     torch.cuda.synchronize()
     assert wush.linear_status(wsp, M, cfg.K, g) == 0
+    if fmt == "nvfp4":
+        assert abs(float(tsw_g[0].item()) - float(ts_w)) <= 2e-7 * float(ts_w)
     Yg = Y[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].cpu().numpy()
     assert rel_fro(Yg, Yo) <= 1e-3

@@ -269,6 +269,23 @@ def test_fixed_transform_variants_run_through_the_same_kernels(kind):
     assert rel_fro(layer(X).cpu().numpy(), Yo) <= 1e-3
 
 
+@pytest.mark.parametrize("g", [16, 32])
+def test_library_fixed_transforms_match_the_oracle(g):
+    """WUSH_KIND_HADAMARD / WUSH_KIND_IDENTITY: the stored bf16 matrix is the oracle's Sylvester-Hadamard matrix
+    (or I) rounded to bf16, the same in every block, and Tinv is the inverse-transpose of the STORED values."""
+    from oracle import wush_transform as WT
+    C = 5
+    for kind, ref in (("hadamard", WT.hadamard(g)), ("identity", np.eye(g))):
+        T, Tinv, info = wush.fixed_transforms(kind, C, g, torch.device("cuda"))
+        torch.cuda.synchronize()
+        assert int(info.abs().max().item()) == 0
+        bits = T.view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(bits, np.broadcast_to(F.f64_to_bf16_bits(ref), (C, g, g)))
+        That = F.bf16_bits_to_f64(bits)
+        want = np.stack([WT.xvsh_from_wush(That[c]) for c in range(C)])
+        assert np.max(np.abs(Tinv.double().cpu().numpy() - want)) <= 1e-6 * np.max(np.abs(want))
+
+
 # ------------------------------------------------------------------ Algorithm 1 on the device
 @pytest.mark.parametrize("fmt,K", [("mxfp4", 1024), ("nvfp4", 512)])
 def test_build_transforms_kernel_against_oracle_and_identities(fmt, K):

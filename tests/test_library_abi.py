@@ -57,6 +57,31 @@ def test_scale_bytes(L):
     assert L.wush_calib_moments_workspace_bytes(512, 2048, 32) % (2048 * 32 * 4) == 0
 
 
+def test_workspace_bytes_covers_every_call(L):
+    for M, N, K, fmt, g in ((128, 2048, 2048, 0, 32), (2048, 4096, 4096, 1, 16), (1, 28672, 8192, 2, 32), (16384, 28672, 8192, 1, 16)):
+        need = L.wush_workspace_bytes(M, N, K, fmt, g)
+        assert need >= L.wush_linear_workspace_bytes(M, K, g) > 0
+        assert need >= L.wush_quantize_weight_workspace_bytes(N, K, fmt, g) > 0
+        assert need >= L.wush_calib_moments_workspace_bytes(N, K, g) > 0
+        assert need >= L.wush_calib_moments_workspace_bytes(M, K, g)
+        assert need == max(L.wush_linear_workspace_bytes(M, K, g), L.wush_quantize_weight_workspace_bytes(N, K, fmt, g),
+                           L.wush_calib_moments_workspace_bytes(max(M, N), K, g))
+    assert L.wush_workspace_bytes(128, 128, 128, 0, 16) == 0        # g does not match the format
+    assert L.wush_workspace_bytes(128, 128, 100, 0, 32) == 0
+    assert L.wush_workspace_bytes(-1, 128, 128, 0, 32) == 0
+
+
+def test_prepare_module_holds_no_arithmetic():
+    """Offline preparation is marshalling only: every matrix it hands to the kernels is made by the library."""
+    import ast
+    src = open(os.path.join(ROOT, "paper_2512_00956_b200", "prepare.py")).read()
+    tree = ast.parse(src)
+    assert not any(isinstance(n, (ast.BinOp, ast.AugAssign, ast.For, ast.While)) and not
+                   (isinstance(n, ast.BinOp) and isinstance(n.op, ast.FloorDiv)) for n in ast.walk(tree))
+    for banned in ("torch.where", "torch.eye", "torch.arange", "math.", "numpy", ".sqrt", "@"):
+        assert banned not in src.split('"""', 2)[2], banned
+
+
 def test_argument_errors_are_found_on_the_host(L):
     p = ctypes.c_void_p(0x1000)         # aligned, never dereferenced: every call below must fail first
     odd = ctypes.c_void_p(0x1004)
@@ -84,6 +109,14 @@ def test_argument_errors_are_found_on_the_host(L):
     assert mo(p, 16, 64, 8, p, p, p, 1 << 20, null) == -3
     assert mo(p, 16, 64, 32, p, null, p, 1 << 20, null) == -1
     assert mo(p, 16, 64, 32, p, p, p, 16, null) == -5
+    assert mo(p, 16, 64, 32, p, odd, p, 1 << 20, null) == -4                    # count not 8-byte aligned
+    assert L.wush_calib_moments_static(p, 16, 64, 32, p, odd, null) == -4
+    bk = L.wush_build_transforms_kind
+    assert bk(null, 0, null, 0, 64, 32, 0.0, 2, null, p, null, null) == -1      # Hadamard: moments optional, outputs not
+    assert bk(null, 0, null, 0, 64, 32, 0.0, 3, p, odd, null, null) == -4
+    assert bk(null, 0, null, 0, 60, 32, 0.0, 2, p, p, null, null) == -2
+    assert bk(null, 0, null, 0, 64, 32, 0.0, 9, p, p, null, null) == -3         # unknown kind
+    assert bk(null, 5, null, 5, 64, 32, 0.0, 0, p, p, null, null) == -1         # WUSH needs the moments
     assert L.wush_quantize_f32(p, 4, 64, 0, 32, null, p, null, 0, null) == -1
     assert L.wush_transform_act_f32(p, 4, 64, p, 24, p, null) == -3
 
