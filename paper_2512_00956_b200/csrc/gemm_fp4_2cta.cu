@@ -142,6 +142,21 @@ __device__ __forceinline__ uint32_t cluster_rank() {
   return r;
 }
 
+// Tile order.  The clusters work on consecutive tile indices at any one time, so the order decides what the L2
+// holds: row-major order makes ~74 concurrent tiles share one 256-row panel of A and touch 74 different panels
+// of B, i.e. the whole of B streams from HBM once per row of tiles.  Here the tiles are walked in bands of
+// RASTER_M tile rows, column by column inside a band: the concurrent tiles then cover RASTER_M panels of A and
+// about 74 / RASTER_M panels of B, and B is read from HBM once per BAND.
+constexpr int RASTER_M = 8;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int per_band = RASTER_M * tiles_n;
+  const int band = tile / per_band, in_band = tile - band * per_band;
+  const int first = band * RASTER_M;
+  const int rows = min(RASTER_M, tiles_m - first);      // the last band may be shorter
+  tn = in_band / rows;
+  tm = first + (in_band - tn * rows);
+}
+
 template <int FMT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
@@ -230,8 +245,10 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     // before the wait, the quantiser's output only after it.  The wait is a no-op for a plain launch.
     const int pre = (cluster_id < num_tiles) ? min(STAGES, num_kb) : 0;
     if (pre > 0) {
-      const int m0 = (cluster_id / tiles_n) * BM + (int)rank * 128;
-      const int n0 = (cluster_id % tiles_n) * BN;
+      int tm, tn;
+      tile_coords(cluster_id, tiles_m, tiles_n, tm, tn);
+      const int m0 = tm * BM + (int)rank * 128;
+      const int n0 = tn * BN;
       if (elect())
         for (int kb = 0; kb < pre; ++kb) weights(kb, kb, n0);
       __syncwarp();
@@ -241,8 +258,10 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
       __syncwarp();
     }
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters) {
-      const int m0 = (tile / tiles_n) * BM + (int)rank * 128;
-      const int n0 = (tile % tiles_n) * BN;
+      int tm, tn;
+      tile_coords(tile, tiles_m, tiles_n, tm, tn);
+      const int m0 = tm * BM + (int)rank * 128;
+      const int n0 = tn * BN;
       for (int kb = (tile == cluster_id ? pre : 0); kb < num_kb; ++kb) {
         g = ((tile - cluster_id) / num_clusters) * num_kb + kb;
         const int s = g % STAGES;
@@ -357,8 +376,10 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
     int it = 0;
     bool ok = true;
     for (int tile = cluster_id; tile < num_tiles && ok; tile += num_clusters, ++it) {
-      const int m0 = (tile / tiles_n) * BM + (int)rank * 128;
-      const int n0 = (tile % tiles_n) * BN + half * 128;
+      int tm, tn;
+      tile_coords(tile, tiles_m, tiles_n, tm, tn);
+      const int m0 = tm * BM + (int)rank * 128;
+      const int n0 = tn * BN + half * 128;
       if (!__all_sync(0xffffffffu, wait(s32(tmem_full), it & 1, abort_flag))) {
         if (lane == 0) { if (*abort_flag == 0 && status) atomicExch(status, 0x140000 | (rank << 15) | (it & 0x7fff)); *abort_flag = 1; }
         ok = false;
