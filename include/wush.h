@@ -238,6 +238,33 @@ int wush_build_transforms_kind(const float* mom_w, int64_t rows_w, const float* 
  * (0 = ok, 3 = singular).  Errors: NULL / SHAPE / FORMAT / ALIGN / CUDA. */
 int wush_invert_transforms(const void* T, int64_t K, int g, float* Tinv, int32_t* info, void* stream);
 
+/* Offline weight preparation, GPTQ case of Algorithm 2: the transforms are built block by block from the UPDATED
+ * weights, and every block's quantisation error is spread first inside the block (the GPTQ subroutine on the
+ * transformed block with the transformed Hessian) and then over all later blocks (W_(j) += L_(j,i) L_(i,i)^-1 E_(i)),
+ * with L L^T the Cholesky factorisation of the inverse of the damped Hessian H + lambda * tr(H)/K * I,
+ * H = Xc^T Xc / B.  Replaces wush_calib_moments + wush_build_transforms + wush_quantize_weight for a layer; the
+ * online calls are the same.
+ *   W      bf16 [N,K];  Xc bf16 [B,K] calibration activations (the layer's inputs).
+ *   lambda damping ratio, > 0 (used for the Hessian and inside Algorithm 1).
+ *   w_tensor_scale  fp32[1] on the device, INPUT, NVFP4 only: the tensor scale has to be fixed before the first
+ *          block is quantised while the weights still change, so the caller chooses it (for example the value
+ *          wush_quantize_weight returns for the same layer); NULL for MXFP4.
+ *   T      bf16 [K/g][g][g] WRITTEN (activation-side transforms, as wush_build_transforms);
+ *   Tinv   fp32 [K/g][g][g] WRITTEN;  codes [N,K/2], scales in layout `sf` WRITTEN.
+ *   info   optional int32[K/g]: 0 ok, 1..3 as wush_build_transforms, 4 = the block's transformed Hessian could not
+ *          be factorised, 5 = the damped Hessian could not be factorised.
+ *   workspace  at least wush_gptq_workspace_bytes(N, K, g) bytes, 256-byte aligned: fp64 copies of W (N x K) and
+ *          of two K x K matrices - about 8 (N K + 2 K^2) bytes.
+ * The scale of a block is fixed when its turn comes, from its current values; each coordinate is rounded to fp32
+ * before it is converted, as in the RTN quantiser.  fp64 arithmetic throughout, fixed summation orders (results
+ * are run-to-run identical).  A sequential offline solver: about 2 K + 6 K/g small kernel launches.
+ * Errors: NULL / SHAPE (incl. lambda <= 0, B <= 0, K > 32768) / FORMAT / ALIGN / WORKSPACE / CUDA. */
+int wush_gptq_quantize_weight(const void* W, int64_t N, int64_t K, const void* Xc, int64_t B,
+                              wush_format_t fmt, int g, float lambda, const float* w_tensor_scale,
+                              void* T, float* Tinv, uint8_t* codes, uint8_t* scales, wush_sf_layout_t sf,
+                              int32_t* info, void* workspace, size_t workspace_bytes, void* stream);
+size_t wush_gptq_workspace_bytes(int64_t N, int64_t K, int g);
+
 /* wush_calib_moments without a workspace argument.  (No counterpart in the paper: this is
  * a packaging variant of the call above, added for hosts where this library must not and
  * cannot obtain device memory at call time - for example a serving process whose allocator

@@ -119,13 +119,19 @@ def propagate_error(Wp, L, i, d, E):
     return Wp
 
 
-def wush_gptq_layer(W_bits, Xc_bits, fmt, lam=0.01, ts_w=None, intra=True):
+def wush_gptq_layer(W_bits, Xc_bits, fmt, lam=0.01, ts_w=None, intra=True, stored_T=None):
     """Algorithm 2, GPTQ case, for one layer.  W_bits [N, K], Xc_bits [B, K] as bf16 bit patterns.
 
     Returns a dict: T_bits uint16 [C,d,d] (bf16 storage of T_wush), T_hat fp64 [C,d,d],
     T_xvsh fp64 [C,d,d], codes uint8 [N, K] (unpacked), scales uint8 [N, C], w_deq fp64 [N, K]
     (dequantised transformed weights, the GEMM operand), W_hat fp64 [N, K] (the quantised layer
-    back in the original space: block i is T_xvsh(i)^-1 W~(i)), ts_w.
+    back in the original space: block i is T_xvsh(i)^-1 W~(i)), ts_w, T_wush fp64 [C,d,d] (Algorithm 1's result
+    before the 16-bit rounding).
+
+    stored_T: optional {block index: uint16 [d,d]} - use these stored transforms for the listed blocks instead
+    of rounding Algorithm 1's result (which is still computed and returned in T_wush).  An entry of T_wush that
+    sits on a bf16 rounding boundary can legitimately be stored either way, and every later block depends on the
+    choice; a comparison with another implementation fixes the choice this way and checks everything else.
     """
     d = Q.GROUP[fmt]
     Wp = F.bf16_bits_to_f64(W_bits).T.copy()             # paper orientation [d_in, d_out]
@@ -139,6 +145,7 @@ def wush_gptq_layer(W_bits, Xc_bits, fmt, lam=0.01, ts_w=None, intra=True):
     L = inverse_hessian_cholesky(Hs, lam)                # Cholesky of the damped Hessian's inverse
     T_bits = np.zeros((C, d, d), dtype=np.uint16)
     T_hat = np.zeros((C, d, d))
+    T_wush = np.zeros((C, d, d))
     T_xvsh = np.zeros((C, d, d))
     codes = np.zeros((d_in, d_out), dtype=np.uint8)
     scales = np.zeros((C, d_out), dtype=np.uint8)
@@ -148,7 +155,10 @@ def wush_gptq_layer(W_bits, Xc_bits, fmt, lam=0.01, ts_w=None, intra=True):
         blk = slice(i * d, (i + 1) * d)
         Wi = Wp[blk]                                     # current (updated) weight block
         M_W = Wi @ Wi.T / d_out                          # second moment of the updated block
-        T_bits[i] = F.f64_to_bf16_bits(WT.wush_block(M_W, M_X[i], lam))    # Algorithm 1, stored in 16 bits
+        T_wush[i] = WT.wush_block(M_W, M_X[i], lam)      # Algorithm 1
+        T_bits[i] = F.f64_to_bf16_bits(T_wush[i])        # stored in 16 bits
+        if stored_T is not None and i in stored_T:
+            T_bits[i] = np.asarray(stored_T[i], dtype=np.uint16)
         T_hat[i] = F.bf16_bits_to_f64(T_bits[i])
         T_xvsh[i] = WT.xvsh_from_wush(T_hat[i]).astype(F32)                # Eq. 6; handed on as fp32, as in the RTN case
         wbar = T_xvsh[i] @ Wi                            # transformed weights
@@ -160,7 +170,7 @@ def wush_gptq_layer(W_bits, Xc_bits, fmt, lam=0.01, ts_w=None, intra=True):
         E = W_hat[blk] - Wi                              # error in the original space
         propagate_error(Wp, L, i, d, E)                  # inter-block error propagation
     return dict(T_bits=T_bits, T_hat=T_hat, T_xvsh=T_xvsh, codes=codes.T.copy(), scales=scales.T.copy(),
-                w_deq=w_deq.T.copy(), W_hat=W_hat.T.copy(), ts_w=ts_w)
+                w_deq=w_deq.T.copy(), W_hat=W_hat.T.copy(), ts_w=ts_w, T_wush=T_wush)
 
 
 def proxy_loss(W_hat, W, Hs):

@@ -16,84 +16,13 @@
 #include "../../include/wush.h"
 #include "wush_device.cuh"
 #include "wush_host.h"
+#include "wush_linalg.cuh"
 
 namespace wush {
 
-constexpr int BT_THREADS = 128;
-
-template <int D>
-__device__ void cholesky_lower(double* A, int* fail) {       // in place; upper triangle zeroed
-  for (int j = 0; j < D; ++j) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      double s = A[j * D + j];
-      for (int k = 0; k < j; ++k) s -= A[j * D + k] * A[j * D + k];
-      if (!(s > 0.0)) { *fail = 1; s = 1.0; }
-      A[j * D + j] = sqrt(s);
-    }
-    __syncthreads();
-    const double piv = A[j * D + j];
-    for (int i = j + 1 + threadIdx.x; i < D; i += BT_THREADS) {
-      double s = A[i * D + j];
-      for (int k = 0; k < j; ++k) s -= A[i * D + k] * A[j * D + k];
-      A[i * D + j] = s / piv;
-    }
-  }
-  __syncthreads();
-  for (int idx = threadIdx.x; idx < D * D; idx += BT_THREADS)
-    if ((idx % D) > (idx / D)) A[idx] = 0.0;
-  __syncthreads();
-}
-
-// Gauss-Jordan with partial pivoting on the D x D matrix Tm (destroyed); Rm becomes the inverse, fac holds D
-// scratch values; the TRANSPOSE of the inverse is written to out (fp32).  *fail = 3 if a pivot is zero.
-template <int D>
-__device__ void inverse_transpose(double* Tm, double* Rm, double* fac_buf, int* perm, int* fail_ptr, float* out) {
-  const int tid = threadIdx.x;
-  for (int idx = tid; idx < D * D; idx += BT_THREADS) Rm[idx] = ((idx / D) == (idx % D)) ? 1.0 : 0.0;
-  __syncthreads();
-  for (int col = 0; col < D; ++col) {
-    if (tid == 0) {
-      int pr = col; double pv = fabs(Tm[col * D + col]);
-      for (int r = col + 1; r < D; ++r) if (fabs(Tm[r * D + col]) > pv) { pv = fabs(Tm[r * D + col]); pr = r; }
-      perm[0] = pr;
-      if (!(pv > 0.0)) *fail_ptr = 3;
-    }
-    __syncthreads();
-    const int pr = perm[0];
-    if (pr != col) {
-      for (int k = tid; k < D; k += BT_THREADS) {
-        double t = Tm[col * D + k]; Tm[col * D + k] = Tm[pr * D + k]; Tm[pr * D + k] = t;
-        t = Rm[col * D + k]; Rm[col * D + k] = Rm[pr * D + k]; Rm[pr * D + k] = t;
-      }
-    }
-    __syncthreads();
-    const double piv = Tm[col * D + col];
-    __syncthreads();
-    for (int k = tid; k < D; k += BT_THREADS) { Tm[col * D + k] /= piv; Rm[col * D + k] /= piv; }
-    __syncthreads();
-    // eliminate column `col` from every other row; factors are read before any row is modified
-    {
-      double* fac = fac_buf;
-      for (int r = tid; r < D; r += BT_THREADS) fac[r] = (r == col) ? 0.0 : Tm[r * D + col];
-      __syncthreads();
-      for (int idx = tid; idx < D * D; idx += BT_THREADS) {
-        const int r = idx / D, k = idx % D;
-        const double f = fac[r];
-        if (f != 0.0) { Tm[idx] -= f * Tm[col * D + k]; Rm[idx] -= f * Rm[col * D + k]; }
-      }
-    }
-    __syncthreads();
-  }
-  for (int idx = tid; idx < D * D; idx += BT_THREADS) {
-    const int j = idx / D, k = idx % D;
-    out[idx] = (float)Rm[k * D + j];      // transpose of the inverse
-  }
-}
-
-template <int D>
+template <int D, typename MT = float>
 __global__ void __launch_bounds__(BT_THREADS)
-build_transforms_kernel(const float* __restrict__ mom_w, double inv_nw, const float* __restrict__ mom_x, double inv_nx,
+build_transforms_kernel(const MT* __restrict__ mom_w, double inv_nw, const MT* __restrict__ mom_x, double inv_nx,
                         double lambda, __nv_bfloat16* __restrict__ T_out, float* __restrict__ Tinv_out,
                         int32_t* __restrict__ info, int with_hadamard) {
   extern __shared__ double sm[];
@@ -108,8 +37,8 @@ build_transforms_kernel(const float* __restrict__ mom_w, double inv_nw, const fl
   __shared__ int perm[D];
   __shared__ int fail, rotated;
   const int c = blockIdx.x, tid = threadIdx.x;
-  const float* mw = mom_w + (size_t)c * D * D;
-  const float* mx = mom_x + (size_t)c * D * D;
+  const MT* mw = mom_w + (size_t)c * D * D;
+  const MT* mx = mom_x + (size_t)c * D * D;
   if (tid == 0) { fail = 0; red[0] = red[1] = 0.0; }
   __syncthreads();
 
@@ -177,7 +106,9 @@ build_transforms_kernel(const float* __restrict__ mom_w, double inv_nw, const fl
           const double u = Jm[r * D + p], v = Jm[r * D + q];
           Jm[r * D + p] = cs * u - sn * v; Jm[r * D + q] = sn * u + cs * v;
         }
-        if (gl == 0 && fabs(ga) > 1e-13 * sqrt(al * be)) rotated = 1;
+        // another sweep while any pair is further from orthogonal than a few rounding errors of its inner product:
+        // the transform's entries inherit this residue divided by the relative gap of neighbouring singular values
+        if (gl == 0 && fabs(ga) > 1e-14 * sqrt(al * be)) rotated = 1;
       }
       __syncthreads();
     }
@@ -312,6 +243,28 @@ cudaError_t run_build_transforms(const float* mom_w, int64_t n_w, const float* m
     build_transforms_kernel<32><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info, wh);
   } else {
     build_transforms_kernel<16><<<C, BT_THREADS, smem, st>>>(mom_w, 1.0 / (double)n_w, mom_x, 1.0 / (double)n_x, lambda, Tb, Tinv, info, wh);
+  }
+  return cudaGetLastError();
+}
+
+// One block from fp64 moment sums (the GPTQ case of Algorithm 2 builds its transforms one at a time from the
+// updated weights): same kernel, double-precision inputs.
+cudaError_t run_build_transform_f64(const double* mom_w, double inv_nw, const double* mom_x, double inv_nx, int g,
+                                    double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st) {
+  const size_t smem = 6 * (size_t)g * g * sizeof(double);
+  __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(T);
+  if (g == 32) {
+    static bool done_of[kDeviceSlots] = {};
+    const int slot = device_slot();
+    if (slot < 0) return cudaErrorInvalidDevice;
+    if (!done_of[slot]) {
+      const cudaError_t e = cudaFuncSetAttribute(build_transforms_kernel<32, double>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      done_of[slot] = true;
+    }
+    build_transforms_kernel<32, double><<<1, BT_THREADS, smem, st>>>(mom_w, inv_nw, mom_x, inv_nx, lambda, Tb, Tinv, info, 1);
+  } else {
+    build_transforms_kernel<16, double><<<1, BT_THREADS, smem, st>>>(mom_w, inv_nw, mom_x, inv_nx, lambda, Tb, Tinv, info, 1);
   }
   return cudaGetLastError();
 }

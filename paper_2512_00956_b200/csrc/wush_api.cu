@@ -292,6 +292,31 @@ int wush_build_transforms(const float* mom_w, int64_t rows_w, const float* mom_x
   return wush_build_transforms_kind(mom_w, rows_w, mom_x, rows_x, K, g, lambda, WUSH_KIND_WUSH, T, Tinv, info, stream);
 }
 
+size_t wush_gptq_workspace_bytes(int64_t N, int64_t K, int g) {
+  if (N <= 0 || K <= 0 || (g != 16 && g != 32) || K % g != 0) return 0;
+  return wush::gptq_workspace_bytes(N, K, g);
+}
+
+int wush_gptq_quantize_weight(const void* W, int64_t N, int64_t K, const void* Xc, int64_t B, wush_format_t fmt, int g,
+                              float lambda, const float* w_tensor_scale, void* T, float* Tinv, uint8_t* codes,
+                              uint8_t* scales, wush_sf_layout_t sf, int32_t* info, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+  int rc = check_fmt(fmt, g);
+  if (rc) return rc;
+  if ((rc = check_shape(N, K, g))) return rc;
+  if (N == 0 || B <= 0 || B > (int64_t)1 << 30 || K > 32768 || !(lambda > 0.0f)) return WUSH_ERR_SHAPE;
+  if (sf != WUSH_SF_LINEAR && sf != WUSH_SF_TILED) return WUSH_ERR_FORMAT;
+  if (!W || !Xc || !T || !Tinv || !codes || !scales || (fmt == WUSH_NVFP4 && !w_tensor_scale)) return WUSH_ERR_NULL;
+  if (!workspace || workspace_bytes < wush_gptq_workspace_bytes(N, K, g)) return WUSH_ERR_WORKSPACE;
+  if (!aligned16(W) || !aligned16(Xc) || !aligned16(T) || !aligned16(Tinv) || !aligned16(codes) || !aligned16(scales) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return WUSH_ERR_ALIGN;
+  const cudaError_t e = wush::run_gptq_quantize_weight(W, N, K, Xc, B, gemm_fmt(fmt), g, (double)lambda, w_tensor_scale, T, Tinv,
+                                                       codes, scales, (int)sf, info, workspace, fmt == WUSH_MXFP4_CEIL ? 1 : 0,
+                                                       (cudaStream_t)stream);
+  return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
+}
+
 int wush_invert_transforms(const void* T, int64_t K, int g, float* Tinv, int32_t* info, void* stream) {
   if (g != 16 && g != 32) return WUSH_ERR_FORMAT;
   if (K <= 0 || K % g != 0) return WUSH_ERR_SHAPE;

@@ -76,6 +76,14 @@ cudaError_t run_invert_transforms(const void* T, int64_t K, int g, float* Tinv, 
 // kind 0: one shared normalised Hadamard matrix, kind 1: the identity, for every block; Tinv = T^-T of the stored values
 cudaError_t run_fixed_transforms(int kind, int64_t K, int g, void* T, float* Tinv, int32_t* info, cudaStream_t st);
 
+cudaError_t run_build_transform_f64(const double* mom_w, double inv_nw, const double* mom_x, double inv_nx, int g,
+                                    double lambda, void* T, float* Tinv, int32_t* info, cudaStream_t st);
+// Algorithm 2, GPTQ case (gptq.cu).  ts_w: NVFP4 weight tensor scale (device, input) or nullptr.
+size_t gptq_workspace_bytes(int64_t N, int64_t K, int g);
+cudaError_t run_gptq_quantize_weight(const void* W, int64_t N, int64_t K, const void* Xc, int64_t B, int fmt, int g,
+                                     double lambda, const float* ts_w, void* T, float* Tinv, uint8_t* codes,
+                                     uint8_t* scales, int sf, int32_t* info, void* workspace, int mx_ceil, cudaStream_t st);
+
 // two-CTA persistent variant (M > 128); cudaErrorNotSupported = use the single-CTA kernel
 int gemm_2cta_cluster_limit(int clusters);   // test hook: 0 = no limit; returns the previous value (per device)
 cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq, const uint8_t* Ws, int64_t M,

@@ -33,10 +33,28 @@ def fixed_transforms(kind, C, d, device):
 class QuantizedLinear:
     """Holds what the online call needs: T, packed W~ codes, TILED scale bytes, tensor scales."""
 
-    def __init__(self, W, Xc, fmt, lam=0.01, transform="wush"):
+    def __init__(self, W, Xc, fmt, lam=0.01, transform="wush", method="rtn"):
+        """method "rtn": the RTN case of Algorithm 2 (moments, transforms, one pass of the weight quantiser);
+        "gptq": its GPTQ case (`wush_gptq_quantize_weight`; NVFP4 takes the RTN case's weight tensor scale)."""
         f, g = wush.FORMATS[fmt]
         self.fmt, self.g = fmt, g
         self.N, self.K = W.shape
+        if method == "gptq":
+            if transform != "wush":
+                raise ValueError("the GPTQ case builds WUSH transforms")
+            ts = None
+            if fmt == "nvfp4":
+                rtn = QuantizedLinear(W, Xc, fmt, lam)
+                ts = rtn.w_tensor_scale
+            self.T, self.Tinv, self.w_codes, self.w_scales, self.info = wush.gptq_quantize_weight(W, Xc, fmt, lam, ts)
+            if int(self.info.abs().max().item()) != 0:
+                raise wush.WushError("wush_gptq_quantize_weight: a factorisation failed (see info)")
+            self.w_tensor_scale = ts
+            self.x_tensor_scale = wush.act_tensor_scale(Xc, self.T, g) if fmt == "nvfp4" else None
+            self._ws = None
+            return
+        if method != "rtn":
+            raise ValueError(method)
         if transform in ("wush", "wus"):
             mom_w, cnt_w = wush.calib_moments(W, g)
             mom_x, cnt_x = wush.calib_moments(Xc, g)

@@ -125,3 +125,19 @@ def weights(cfg, N=None, K=None, chunk=2048):
 def layer_inputs(cfg, M=None, N=None, K=None, B=None):
     """All three tensors of one layer; sizes may be shrunk for quick tests."""
     return dict(X=activations(cfg, M, K), W=weights(cfg, N, K), Xc=calibration(cfg, B, K))
+
+
+def correlated_layer(seed, N, K, B, rho=0.6):
+    """(W bits [N, K], Xc bits [B, K]) with activations correlated ACROSS quantisation blocks: an AR(1) chain over
+    the channels plus a component shared by all channels, then log-normal channel scales.  Stand-in for a layer
+    whose Hessian is far from block diagonal (the case error propagation between blocks is for)."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    z = rng.standard_normal((B, K))
+    x = np.empty_like(z)
+    x[:, 0] = z[:, 0]
+    for k in range(1, K):
+        x[:, k] = rho * x[:, k - 1] + np.sqrt(1.0 - rho * rho) * z[:, k]
+    x += 0.5 * rng.standard_normal((B, 1))
+    x *= np.exp(0.5 * rng.standard_normal(K))[None, :]
+    w = 0.02 * rng.standard_normal((N, K))
+    return to_bf16_bits(w), to_bf16_bits(x)

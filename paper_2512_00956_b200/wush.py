@@ -28,6 +28,7 @@ EXPORTS = [
     "wush_build_transforms", "wush_quantize_act_dynamic", "wush_check_division", "wush_debug_gemm_clusters",
     "wush_debug_drop_tile", "wush_decode_status", "wush_build_transforms_kind", "wush_invert_transforms",
     "wush_act_tensor_scale", "wush_workspace_bytes", "wush_debug_quantiser_rows",
+    "wush_gptq_quantize_weight", "wush_gptq_workspace_bytes",
 ]
 STATIC_SCRATCH_BYTES = 4 << 20
 
@@ -60,6 +61,10 @@ def lib():
         L.wush_linear.argtypes = [vp, i64, i64, vp, vp, vp, i64, vp, vp, i32, i32, vp, i32, vp, sz, vp]
         L.wush_linear_workspace_bytes.restype = sz
         L.wush_linear_workspace_bytes.argtypes = [i64, i64, i32]
+        L.wush_gptq_workspace_bytes.restype = sz
+        L.wush_gptq_workspace_bytes.argtypes = [i64, i64, i32]
+        L.wush_gptq_quantize_weight.restype = i32
+        L.wush_gptq_quantize_weight.argtypes = [vp, i64, i64, vp, i64, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp]
         L.wush_workspace_bytes.restype = sz
         L.wush_workspace_bytes.argtypes = [i64, i64, i64, i32, i32]
         L.wush_debug_quantiser_rows.argtypes = [i32]
@@ -276,6 +281,26 @@ def build_transforms(mom_w, rows_w, mom_x, rows_x, g, lam=0.01, kind="wush"):
     check(lib().wush_build_transforms_kind(_ptr(mom_w), int(rows_w), _ptr(mom_x), int(rows_x), K, g, float(lam),
                                            KINDS[kind], _ptr(T), _ptr(Tinv), _ptr(info), _stream()))
     return T, Tinv, info[:C]
+
+
+def gptq_quantize_weight(W, Xc, fmt, lam=0.01, w_tensor_scale=None, sf=SF_TILED):
+    """Algorithm 2, GPTQ case (wush_gptq_quantize_weight).  W bf16 [N,K], Xc bf16 [B,K] ->
+    (T bf16 [K/g,g,g], Tinv fp32 [K/g,g,g], codes, scale bytes, info int32 [K/g]).  NVFP4 needs w_tensor_scale (fp32, device)."""
+    f, g = _fmt(fmt)
+    _dev(W, Xc, w_tensor_scale)
+    N, K = W.shape
+    C = K // g
+    T = torch.empty((C, g, g), dtype=torch.bfloat16, device=W.device)
+    Tinv = torch.empty((C, g, g), dtype=torch.float32, device=W.device)
+    codes, scales = _alloc_q(N, K, g, sf, W.device)
+    info = torch.zeros(max(C, 4), dtype=torch.int32, device=W.device)
+    nws = lib().wush_gptq_workspace_bytes(N, K, g)
+    ws = torch.empty(nws + 256, dtype=torch.uint8, device=W.device)
+    off = (-ws.data_ptr()) % 256
+    check(lib().wush_gptq_quantize_weight(_ptr(W), N, K, _ptr(Xc), Xc.shape[0], f, g, float(lam), _ptr(w_tensor_scale),
+                                          _ptr(T), _ptr(Tinv), _ptr(codes), _ptr(scales), sf, _ptr(info),
+                                          ctypes.c_void_p(ws.data_ptr() + off), nws, _stream()))
+    return T, Tinv, codes, scales, info[:C]
 
 
 def invert_transforms(T, g):

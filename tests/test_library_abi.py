@@ -117,6 +117,15 @@ def test_argument_errors_are_found_on_the_host(L):
     assert bk(null, 0, null, 0, 60, 32, 0.0, 2, p, p, null, null) == -2
     assert bk(null, 0, null, 0, 64, 32, 0.0, 9, p, p, null, null) == -3         # unknown kind
     assert bk(null, 5, null, 5, 64, 32, 0.0, 0, p, p, null, null) == -1         # WUSH needs the moments
+    gq = L.wush_gptq_quantize_weight
+    big = L.wush_gptq_workspace_bytes(16, 64, 32)
+    assert big >= 8 * (16 * 64 + 2 * 64 * 64)
+    wsp = ctypes.c_void_p(0x10000)
+    assert gq(p, 16, 64, p, 8, 0, 32, 0.0, null, p, p, p, p, 0, null, wsp, big, null) == -2      # lambda must be positive
+    assert gq(p, 16, 64, p, 0, 0, 32, 0.01, null, p, p, p, p, 0, null, wsp, big, null) == -2     # no calibration tokens
+    assert gq(p, 16, 64, p, 8, 1, 16, 0.01, null, p, p, p, p, 0, null, wsp, big, null) == -1     # NVFP4 needs the tensor scale
+    assert gq(p, 16, 64, p, 8, 0, 32, 0.01, null, p, p, p, p, 0, null, wsp, big - 1, null) == -5
+    assert gq(p, 16, 64, p, 8, 0, 32, 0.01, null, p, p, p, p, 0, null, ctypes.c_void_p(0x10010), big, null) == -4
     assert L.wush_quantize_f32(p, 4, 64, 0, 32, null, p, null, 0, null) == -1
     assert L.wush_transform_act_f32(p, 4, 64, p, 24, p, null) == -3
 

@@ -26,19 +26,8 @@ from oracle import wush_transform as WT
 from paper_2512_00956_b200 import synth
 
 
-def _correlated_layer(seed, N, K, B, rho=0.6):
-    """Weights and calibration tokens whose channels are correlated ACROSS blocks (AR(1) mixing plus a shared
-    component), so that inter-block propagation has something to do."""
-    rng = np.random.default_rng(seed)
-    z = rng.standard_normal((B, K))
-    x = np.empty_like(z)
-    x[:, 0] = z[:, 0]
-    for k in range(1, K):
-        x[:, k] = rho * x[:, k - 1] + np.sqrt(1 - rho * rho) * z[:, k]
-    x += 0.5 * rng.standard_normal((B, 1))
-    x *= np.exp(0.5 * rng.standard_normal(K))[None, :]
-    W = 0.02 * rng.standard_normal((N, K))
-    return F.f64_to_bf16_bits(W), F.f64_to_bf16_bits(x)
+def _correlated_layer(seed, N, K, B):
+    return synth.correlated_layer(seed, N, K, B)
 
 
 def test_inverse_hessian_cholesky_identity():
