@@ -297,12 +297,15 @@ int wush_calib_moments_static(const void* Xc, int64_t B, int64_t K, int g, float
 int wush_quantize_f32(const float* V, int64_t R, int64_t K, wush_format_t fmt, int g,
                       const float* tensor_scale, uint8_t* codes, uint8_t* scales,
                       wush_sf_layout_t sf, void* stream);
-/* The NVFP4 scale byte needs (AbsMax / 6) / tensor_scale with both divisions correctly rounded.  Inside
- * AbsMax in [2^-50, 2^50] and tensor_scale in [2^-40, 2^40] the kernels evaluate them without the IEEE
- * division sequence (reciprocal of the divisor, two fused multiply-add corrections); outside they use the
- * IEEE division.  This call checks the equivalence on the device: for each of the n divisors b (fp32, device
- * array, normal, in [2^-40, 2^40]) it compares the two for EVERY fp32 x in [2^-60, 2^60] and stores the number
- * of x that differ in mismatches[i] (uint64, device array; expected: all zero).  About 1 ms per divisor. */
+/* The NVFP4 scale byte is E4M3((AbsMax / 6) / tensor_scale) with both divisions correctly rounded.  The kernels
+ * take two shortcuts that must give the same byte: (a) inside AbsMax in [2^-50, 2^50] and tensor_scale in
+ * [2^-40, 2^40] the divisions are evaluated without the IEEE division sequence (reciprocal of the divisor, two
+ * fused multiply-add corrections); (b) where AbsMax * RN(1 / (6 tensor_scale)) is clear of every E4M3 rounding
+ * boundary by more than its own error, that product is converted directly.  This call checks both on the device:
+ * for each of the n values b (fp32, device array, normal, in [2^-40, 2^40]) it compares, for EVERY fp32 x in
+ * [2^-60, 2^60], x / b by (a) with the IEEE quotient, and the scale byte of a block with AbsMax = x under tensor
+ * scale b as the kernels compute it with the byte of the IEEE sequence; mismatches[i] (uint64, device array)
+ * receives the number of x for which either differs (expected: all zero).  A few ms per value. */
 int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void* stream);
 /* Test hook for the persistent GEMM (M > 128): use at most `clusters` two-CTA clusters in later calls on the
  * current device (0 = as many as fit, the default; the setting is per device, shared by all threads).  With few clusters even a small problem

@@ -123,25 +123,42 @@ __device__ __forceinline__ float div_rn_fma(float x, float b, float y) {
   return __fmaf_rn(r, y, q);
 }
 constexpr float kRcp6 = 0.16666667163372040f;        // RN(1/6) = 0x3E2AAAAB
-// Per-kernel constants of the fast scale path: rts = RN(1 / ts), usable while ts lies in [2^-40, 2^40]
+// Per-kernel constants of the fast scale paths: rts = RN(1 / ts) and c = RN(RN(1/6) * rts) ~ 1 / (6 ts), usable
+// while ts lies in [2^-40, 2^40]
 struct NvScaleFast {
-  float ts, rts;
+  float ts, rts, c;
   bool ts_ok;
 };
 __device__ __forceinline__ NvScaleFast nv_scale_fast(float t) {
   NvScaleFast f;
   f.ts = t;
   f.rts = __frcp_rn(t);
+  f.c = __fmul_rn(kRcp6, f.rts);
   f.ts_ok = (t >= 0x1p-40f && t <= 0x1p40f);
   return f;
 }
-// The same byte as nv_scale_byte(amax, f.ts): blocks with amax in [2^-50, 2^50] take the FMA divisions (both
-// intermediates then stay far inside the normal range), everything else - zero blocks included - the IEEE ones.
-__device__ __forceinline__ uint32_t nv_scale_byte(float amax, const NvScaleFast& f) {
+// The pinned sequence with the divisions done by FMAs where that is exact (blocks with amax in [2^-50, 2^50], both
+// intermediates then stay far inside the normal range), the IEEE ones otherwise - zero blocks included.
+__device__ __forceinline__ uint32_t nv_scale_byte_slow(float amax, const NvScaleFast& f) {
   float r;
   if (f.ts_ok && amax >= 0x1p-50f && amax <= 0x1p50f) r = div_rn_fma(div_rn_fma(amax, 6.0f, kRcp6), f.ts, f.rts);
   else r = __fdiv_rn(__fdiv_rn(amax, 6.0f), f.ts);
   return static_cast<uint32_t>(__nv_cvt_float_to_fp8(r, __NV_SATFINITE, __NV_E4M3));
+}
+// The same byte as nv_scale_byte(amax, f.ts).  The byte only depends on which E4M3 rounding interval r falls into, so
+// an approximation of r decides it whenever it is clear of every interval boundary: r' = RN(amax * c) lies within
+// 4 ulp of the pinned r (c carries 1.5 ulp, the product half an ulp, the pinned r one ulp against the exact
+// quotient).  In the normal range of E4M3 (r >= 2^-6) the boundaries are the values whose low 20 mantissa bits
+// are 0x80000; r' further than 16 ulp from that pattern gives the pinned byte by conversion (above 448 everything
+// saturates, and the boundaries 432 and 464 on the way there have the same pattern).  Anything else - about one
+// block in 30000, the subnormal range, zero blocks - takes the pinned sequence.  wush_check_division compares the
+// two for every fp32 amax.
+__device__ __forceinline__ uint32_t nv_scale_byte(float amax, const NvScaleFast& f) {
+  const float rf = __fmul_rn(amax, f.c);
+  const uint32_t low = __float_as_uint(rf) & 0xFFFFFu;
+  if (f.ts_ok && rf >= 0x1.01p-6f && (low - 0x7FFF0u) >= 0x20u)
+    return static_cast<uint32_t>(__nv_cvt_float_to_fp8(rf, __NV_SATFINITE, __NV_E4M3));
+  return nv_scale_byte_slow(amax, f);
 }
 __device__ __forceinline__ float nv_mult_of_byte(uint32_t byte, float ts) {
   const float d = __fmul_rn(e4m3_to_float(byte), ts);
