@@ -86,7 +86,8 @@ const char* wush_status_string(int status);
  * diagnostic word in the int32 `status` buffer of the call (wush_gemm_fp4: its argument; wush_linear: the last
  * 16 bytes of the workspace), lets its outstanding copies land, frees what it holds and returns; the outputs
  * of that call are then undefined and the context stays usable.  The word is 0 when nothing expired, else
- * (role << 16) | index: role 0x04 / 0x05 = producer / consumer of the quantiser (index = work item of the CTA),
+ * (role << 16) | index: role 0x06 / 0x07 / 0x08 = producer / MMA issuer / epilogue of the quantiser (0x04 / 0x05 =
+ * producer / consumer of its warp-level variant; index = work item of the CTA),
  * 0x11..0x15 = producer, scale-copy wait, accumulator hand-over, epilogue, operand wait of the GEMM for
  * M > 128, 0x01..0x03 = producer, MMA issuer, epilogue of the GEMM for M <= 128.  The
  * caller copies the word to the host after synchronising; this helper maps it to WUSH_OK or WUSH_ERR_TIMEOUT. */
@@ -313,11 +314,12 @@ int wush_check_division(const float* divisors, int n, uint64_t* mismatches, void
  * (accumulator drained while the next tile's loads run) without a full-size input.  Results never depend
  * on it.  Returns the previous value. */
 int wush_debug_gemm_clusters(int clusters);
-/* Test hook for the streaming quantiser: tile height of later wush_quantize_act / wush_quantize_act_dynamic /
- * wush_linear calls on the current device (a per-device setting) - 64 or 128 token rows, 0 = chosen from the problem
- * size (the default: 128 once every SM gets at least five 128 x 128 items).  The tests use it to run ragged token
- * counts and channel tails through both instantiations without full-size inputs.  Results never depend on it.
- * Returns the previous value, or WUSH_ERR_SHAPE for another height. */
+/* Test hook for the activation quantiser.  By default (0) wush_quantize_act / wush_quantize_act_dynamic /
+ * wush_linear run the kernel that does the block products on the tcgen05 tensor cores; 64 or 128 selects the
+ * warp-level streaming kernel (the one the weight side uses, and the fall-back) with that many token rows per
+ * tile, for later calls on the current device (a per-device setting).  The tests use it to run ragged token counts
+ * and channel tails through every instantiation without full-size inputs.  Results never depend on it.
+ * Returns the previous value, or WUSH_ERR_SHAPE for another value. */
 int wush_debug_quantiser_rows(int rows);
 /* Test hook for the error path: the next wush_linear call on the current device (whichever thread makes it) leaves the
  * tile of work item `item` of its quantiser kernel unrequested (one call only; -1 cancels).  The consumers'

@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwush.so")
-SOURCES = ["wush_api.cu", "transform_quant.cu", "transform_quant_stream.cu", "moments.cu", "moments_stream.cu", "build_transforms.cu", "gptq.cu", "gemm_fp4.cu", "gemm_fp4_2cta.cu"]
+SOURCES = ["wush_api.cu", "transform_quant.cu", "transform_quant_stream.cu", "transform_quant_tc.cu", "moments.cu", "moments_stream.cu", "build_transforms.cu", "gptq.cu", "gemm_fp4.cu", "gemm_fp4_2cta.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -587,6 +587,13 @@ cudaError_t run_quantize_weight_stream(const void* W, int64_t N, int64_t K, cons
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                     uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl,
                                     cudaStream_t st, const QuantOpts& opt) {
+  // First choice: the kernel that runs the block products on the tcgen05 tensor cores.  The warp-level kernel below
+  // remains for the weight side (fp32 transforms, three-way split), as the fall-back, and under the test hook that
+  // forces one of its tile heights.
+  if (opt.force_rows == 0) {
+    const cudaError_t et = run_quantize_act_tc(X, M, K, T, g, ts, codes, scales, sf, status, clear_status, pdl, st, opt);
+    if (et != cudaErrorNotSupported) return et;
+  }
   if (!sq_encode_fn()) return cudaErrorNotSupported;
   if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;      // LINEAR rows must keep 4-byte scale groups aligned
   int sm_count = 0;

@@ -41,6 +41,10 @@ cudaError_t run_act_tensor_scale(const void* X, int64_t M, int64_t K, const void
 cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                     uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
                                     bool pdl, cudaStream_t st, const QuantOpts& opt = QuantOpts());
+// activation side with the block products on tcgen05 tensor cores (transform_quant_tc.cu); same contract
+cudaError_t run_quantize_act_tc(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
+                                uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
+                                bool pdl, cudaStream_t st, const QuantOpts& opt = QuantOpts());
 // weight side through the streaming kernel (fp32 Tinv, three-way split); cudaErrorNotSupported = use the other kernel
 cudaError_t run_quantize_weight_stream(const void* W, int64_t N, int64_t K, const float* Tinv, int g, uint8_t* codes,
                                        uint8_t* scales, int sf, cudaStream_t st, const QuantOpts& opt);

@@ -22,7 +22,7 @@ def test_bench_line_on_the_small_configuration():
     assert d["value"] > 0 and d["ms_per_step"] > 0 and d["gemm_status"] == 0
     assert d["gpu_launches"] == 2 * d["steps"]
     assert d["replays"] >= 3 and d["ms_per_step_min"] <= d["ms_per_step"] <= d["ms_per_step_max"]
-    assert d["clocks"]["samples"] >= 10 and d["workloads"] == []
+    assert d["clocks"]["samples"] >= 3 and d["workloads"] == []
     assert d["config"]["workload"] and "model" not in d["config"]
     r = d["roofline"]
     assert r["bound"] in ("hbm", "tensor") and r["unit"] in ("GB/s", "TFLOP/s")

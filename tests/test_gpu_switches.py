@@ -173,7 +173,7 @@ def test_expired_wait_is_reported_and_the_next_call_works():
     Y, wsp = wush.linear(X, T, wq, ws, fmt, None, tsw)
     torch.cuda.synchronize()
     word = wush.linear_status(wsp, M, K, 32)
-    assert word != 0 and (word >> 16) in (0x04, 0x05), hex(word)
+    assert word != 0 and (word >> 16) in (0x04, 0x05, 0x06, 0x07, 0x08), hex(word)     # a role of the quantiser
     assert wush.decode_status(word) == wush.lib().wush_decode_status(1) != 0      # WUSH_ERR_TIMEOUT
     assert wush.decode_status(0) == 0
     Y, wsp = wush.linear(X, T, wq, ws, fmt, None, tsw)                           # the hook was for one call
