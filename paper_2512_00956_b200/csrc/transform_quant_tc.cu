@@ -137,6 +137,23 @@ __device__ __forceinline__ uint32_t quantise_block(const uint32_t* u, int mx_cei
   return byte;
 }
 
+// The transforms of one 128-channel panel as B operands, one tile per 64-channel box: row j = 128 bytes = the j-th
+// rows of the box's 64 / G blocks side by side; 16-byte chunk c of row j sits at chunk c ^ (j & 7) (128-byte swizzle,
+// as TMA writes the A operand).  Thread `tid` of `nthreads` copies its share; the caller fences and synchronises.
+template <int G>
+__device__ __forceinline__ void copy_transforms(const __nv_bfloat16* __restrict__ T, int panel, int nsub, uint8_t* tdst0, int tid, int nthreads) {
+  constexpr int BLOCKS = 64 / G;
+  constexpr int CHUNKS = G * 8;                        // 16-byte chunks of a tile: G rows x 8
+  constexpr int CPB = G / 8;                           // chunks per block row (64 B or 32 B)
+  for (int q = tid; q < nsub * CHUNKS; q += nthreads) {
+    const int sub = q / CHUNKS, qq = q % CHUNKS;
+    const int j = qq >> 3, c = qq & 7;
+    const int blk = (panel * SUBS + sub) * BLOCKS + c / CPB;
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(T + ((int64_t)blk * G + j) * G + (c % CPB) * 8));
+    *reinterpret_cast<uint4*>(tdst0 + sub * TSUB_BYTES + j * 128 + ((c ^ (j & 7)) << 4)) = v;
+  }
+}
+
 // AMAX = true: the same walk and the same products, but only the AbsMax of everything computed is folded into
 // *ts_out (bit pattern of a non-negative float, atomicMax): first pass of the per-batch NVFP4 tensor scale.
 template <int G, bool AMAX>
@@ -191,6 +208,17 @@ tq_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __re
     if (nv_dynamic && blockIdx.x == 0 && threadIdx.x == 0 && ts_out != nullptr) *ts_out = ts;
     __syncthreads();
   }
+  // the transforms of the CTA's first STAGES items, copied by all threads at once (later changes of panel - rare, see
+  // the grid's size - are the producer warp's job)
+  for (int s = 0; s < STAGES; ++s) {
+    const int it = blockIdx.x + s * gridDim.x;
+    if (it >= num_items) break;
+    const int panel = it % num_panels;
+    copy_transforms<G>(T, panel, min(SUBS, (int)(K >> 6) - panel * SUBS), smem + s * STAGE_BYTES + X_BYTES, threadIdx.x, THREADS);
+    if (threadIdx.x == 0) stage_tag[s] = panel;
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // Items are numbered row-block-major (item = row block * panels + panel) and dealt out round-robin, CTA c taking
@@ -223,22 +251,8 @@ tq_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __re
               ::"r"(s32(stage + sub * BOX_BYTES)), "l"(&mapX), "r"((panel * SUBS + sub) * 64), "r"(rb * ROWS), "r"(bar) : "memory");
       }
       __syncwarp();
-      if (stage_tag[s] != panel) {
-        // the panel's transforms as B operands, one tile per 64-channel box: row j = 128 bytes = the j-th rows of the
-        // box's 64 / G blocks side by side; 16-byte chunk c of row j sits at chunk c ^ (j & 7) (128-byte swizzle, as
-        // TMA writes the A operand)
-        constexpr int CHUNKS = G * 8;                        // 16-byte chunks of a tile: G rows x 8
-        constexpr int CPB = G / 8;                           // chunks per block row (64 B or 32 B)
-        for (int sub = 0; sub < nsub; ++sub) {
-          uint8_t* tdst = stage + X_BYTES + sub * TSUB_BYTES;
-#pragma unroll
-          for (int q = lane; q < CHUNKS; q += 32) {
-            const int j = q >> 3, c = q & 7;
-            const int blk = (panel * SUBS + sub) * BLOCKS + c / CPB;
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(T + ((int64_t)blk * G + j) * G + (c % CPB) * 8));
-            *reinterpret_cast<uint4*>(tdst + j * 128 + ((c ^ (j & 7)) << 4)) = v;
-          }
-        }
+      if (stage_tag[s] != panel) {                                     // (the first STAGES items were prepared at entry)
+        copy_transforms<G>(T, panel, nsub, stage + X_BYTES, lane, 32);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // written by threads, read by the tensor core
         __syncwarp();
         if (lane == 0) stage_tag[s] = panel;
