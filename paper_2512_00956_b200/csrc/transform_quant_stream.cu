@@ -590,7 +590,9 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
   // First choice: the kernel that runs the block products on the tcgen05 tensor cores.  The warp-level kernel below
   // remains for the weight side (fp32 transforms, three-way split), as the fall-back, and under the test hook that
   // forces one of its tile heights.
-  if (opt.force_rows == 0) {
+  // (decode-sized batches stay on the warp-level kernel: a launch with a handful of 128-row items is dominated by
+  // set-up, and that kernel has 1-2 us less of it - no tensor-memory allocation, a third of the threads)
+  if (opt.force_rows == 0 && M > 256) {
     const cudaError_t et = run_quantize_act_tc(X, M, K, T, g, ts, codes, scales, sf, status, clear_status, pdl, st, opt);
     if (et != cudaErrorNotSupported) return et;
   }
