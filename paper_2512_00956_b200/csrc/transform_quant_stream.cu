@@ -574,6 +574,10 @@ static cudaError_t stream_sm_count(int* out) {
 // the AbsMax pass / tensor-scale pointers for NVFP4 exactly as on the activation side.
 cudaError_t run_quantize_weight_stream(const void* W, int64_t N, int64_t K, const float* Tinv, int g, uint8_t* codes,
                                        uint8_t* scales, int sf, cudaStream_t st, const QuantOpts& opt) {
+  if (opt.force_rows == 0 && N > 256) {          // first choice: the tcgen05 kernel (as on the activation side)
+    const cudaError_t et = run_quantize_weight_tc(W, N, K, Tinv, g, codes, scales, sf, st, opt);
+    if (et != cudaErrorNotSupported) return et;
+  }
   if (!sq_encode_fn()) return cudaErrorNotSupported;
   if (sf == 0 && ((K / g) & 3) != 0) return cudaErrorNotSupported;
   int sm_count = 0;

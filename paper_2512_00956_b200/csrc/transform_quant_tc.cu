@@ -37,16 +37,18 @@ constexpr int ROWS = 128;
 constexpr int SUBS = 2;                        // 64-channel boxes per item: rows are read 256 contiguous bytes at a time
 constexpr int BOX_BYTES = ROWS * 128;          // 128 rows x 64 bf16 channels
 constexpr int X_BYTES = SUBS * BOX_BYTES;
-constexpr int TSUB_BYTES = 4096;               // transforms of one 64-channel box as a B operand
-constexpr int T_BYTES = SUBS * TSUB_BYTES;
-constexpr int STAGE_BYTES = X_BYTES + T_BYTES;
+constexpr int TSUB_BYTES = 4096;               // transforms of one 64-channel box as a B operand (one bf16 term)
 constexpr int STAGES = 8 / SUBS;
+// NSPLIT = 1: bf16 transforms (activations).  NSPLIT = 3: fp32 transforms (weight side) split exactly into three bf16
+// terms lo + mid + hi, one B tile each; the three products are accumulated smallest first in the same accumulator.
+__host__ __device__ constexpr int t_bytes(int nsplit) { return SUBS * nsplit * TSUB_BYTES; }
+__host__ __device__ constexpr int stage_bytes(int nsplit) { return X_BYTES + t_bytes(nsplit); }
 constexpr int EPI_WARPS = 16;                  // four groups of four
 constexpr int THREADS = (2 + EPI_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int ACC_COLS = SUBS * 64;
 // ring | full[8] empty[8] tfull[8] tempty[8] (256 B) | tmem slot, abort flag, stage tags (64 B) | NVFP4 multiplier table (512 B)
-constexpr int SMEM = 1024 + STAGES * STAGE_BYTES + 256 + 64 + 512;
+__host__ __device__ constexpr int smem_bytes(int nsplit) { return 1024 + STAGES * stage_bytes(nsplit) + 256 + 64 + 512; }
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
@@ -140,8 +142,8 @@ __device__ __forceinline__ uint32_t quantise_block(const uint32_t* u, int mx_cei
 // The transforms of one 128-channel panel as B operands, one tile per 64-channel box: row j = 128 bytes = the j-th
 // rows of the box's 64 / G blocks side by side; 16-byte chunk c of row j sits at chunk c ^ (j & 7) (128-byte swizzle,
 // as TMA writes the A operand).  Thread `tid` of `nthreads` copies its share; the caller fences and synchronises.
-template <int G>
-__device__ __forceinline__ void copy_transforms(const __nv_bfloat16* __restrict__ T, int panel, int nsub, uint8_t* tdst0, int tid, int nthreads) {
+template <int G, int NSPLIT>
+__device__ __forceinline__ void copy_transforms(const void* __restrict__ Tsrc, int panel, int nsub, uint8_t* tdst0, int tid, int nthreads) {
   constexpr int BLOCKS = 64 / G;
   constexpr int CHUNKS = G * 8;                        // 16-byte chunks of a tile: G rows x 8
   constexpr int CPB = G / 8;                           // chunks per block row (64 B or 32 B)
@@ -149,20 +151,48 @@ __device__ __forceinline__ void copy_transforms(const __nv_bfloat16* __restrict_
     const int sub = q / CHUNKS, qq = q % CHUNKS;
     const int j = qq >> 3, c = qq & 7;
     const int blk = (panel * SUBS + sub) * BLOCKS + c / CPB;
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(T + ((int64_t)blk * G + j) * G + (c % CPB) * 8));
-    *reinterpret_cast<uint4*>(tdst0 + sub * TSUB_BYTES + j * 128 + ((c ^ (j & 7)) << 4)) = v;
+    const int64_t src = ((int64_t)blk * G + j) * G + (c % CPB) * 8;           // first of this chunk's 8 entries
+    uint8_t* dst = tdst0 + sub * NSPLIT * TSUB_BYTES + j * 128 + ((c ^ (j & 7)) << 4);
+    if (NSPLIT == 1) {
+      *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(Tsrc) + src));
+    } else {
+      const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(Tsrc) + src);
+      const float4 v0 = __ldg(p), v1 = __ldg(p + 1);
+      const float f[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+      uint32_t pk[3][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint32_t h[2][3];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const float x = f[2 * i + e];
+          const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+          const float r1 = x - __bfloat162float(hi);               // exact
+          const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+          const float r2 = r1 - __bfloat162float(mid);              // exact
+          const __nv_bfloat16 lo = __float2bfloat16_rn(r2);
+          h[e][0] = __bfloat16_as_ushort(lo); h[e][1] = __bfloat16_as_ushort(mid); h[e][2] = __bfloat16_as_ushort(hi);
+        }
+#pragma unroll
+        for (int sp = 0; sp < 3; ++sp) pk[sp][i] = h[0][sp] | (h[1][sp] << 16);
+      }
+#pragma unroll
+      for (int sp = 0; sp < 3; ++sp)                      // tile 0 = lo, 1 = mid, 2 = hi
+        *reinterpret_cast<uint4*>(dst + sp * TSUB_BYTES) = make_uint4(pk[sp][0], pk[sp][1], pk[sp][2], pk[sp][3]);
+    }
   }
 }
 
 // AMAX = true: the same walk and the same products, but only the AbsMax of everything computed is folded into
 // *ts_out (bit pattern of a non-negative float, atomicMax): first pass of the per-batch NVFP4 tensor scale.
-template <int G, bool AMAX>
+template <int G, bool AMAX, int NSPLIT = 1>
 __global__ void __launch_bounds__(THREADS, 1)
-tq_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __restrict__ T, int64_t M, int64_t K,
+tq_tc_kernel(const __grid_constant__ CUtensorMap mapX, const void* __restrict__ T, int64_t M, int64_t K,
              const float* __restrict__ ts_ptr, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales, int sf_layout,
              int num_panels, int num_items, int32_t* __restrict__ status, int clear_status,
              const uint32_t* __restrict__ amax_in, float* __restrict__ ts_out, int mx_ceil, int drop_item) {
-  constexpr int BLOCKS = 64 / G;                     // quantisation blocks per item row: 2 (g = 32) or 4 (g = 16)
+  constexpr int BLOCKS = 64 / G;                     // quantisation blocks per box row: 2 (g = 32) or 4 (g = 16)
+  constexpr int STAGE_BYTES = stage_bytes(NSPLIT);
   extern __shared__ uint8_t raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
@@ -214,7 +244,7 @@ tq_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __re
     const int it = blockIdx.x + s * gridDim.x;
     if (it >= num_items) break;
     const int panel = it % num_panels;
-    copy_transforms<G>(T, panel, min(SUBS, (int)(K >> 6) - panel * SUBS), smem + s * STAGE_BYTES + X_BYTES, threadIdx.x, THREADS);
+    copy_transforms<G, NSPLIT>(T, panel, min(SUBS, (int)(K >> 6) - panel * SUBS), smem + s * STAGE_BYTES + X_BYTES, threadIdx.x, THREADS);
     if (threadIdx.x == 0) stage_tag[s] = panel;
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -252,7 +282,7 @@ tq_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __re
       }
       __syncwarp();
       if (stage_tag[s] != panel) {                                     // (the first STAGES items were prepared at entry)
-        copy_transforms<G>(T, panel, nsub, stage + X_BYTES, lane, 32);
+        copy_transforms<G, NSPLIT>(T, panel, nsub, stage + X_BYTES, lane, 32);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // written by threads, read by the tensor core
         __syncwarp();
         if (lane == 0) stage_tag[s] = panel;
@@ -289,14 +319,17 @@ tq_tc_kernel(const __grid_constant__ CUtensorMap mapX, const __nv_bfloat16* __re
         const int nsub = min(SUBS, (int)(K >> 6) - panel * SUBS);
         for (int sub = 0; sub < nsub; ++sub) {
           const uint64_t adesc = op_desc(s32(smem + s * STAGE_BYTES + sub * BOX_BYTES));
-          const uint64_t bdesc = op_desc(s32(smem + s * STAGE_BYTES + X_BYTES + sub * TSUB_BYTES));
           const uint32_t d = tmem_base + s * ACC_COLS + sub * 64;
 #pragma unroll
           for (int b = 0; b < BLOCKS; ++b) {
 #pragma unroll
-            for (int ks = 0; ks < G / 16; ++ks) {            // 16 channels (32 bytes) per instruction
-              const uint32_t off = (uint32_t)(b * 2 * G + ks * 32) >> 4;
-              mma_bf16(d + b * G, adesc + off, bdesc + off, idesc, ks);
+            for (int sp = 0; sp < NSPLIT; ++sp) {            // lo, mid, hi term of the transform (one term for bf16 transforms)
+              const uint64_t bdesc = op_desc(s32(smem + s * STAGE_BYTES + X_BYTES + (sub * NSPLIT + sp) * TSUB_BYTES));
+#pragma unroll
+              for (int ks = 0; ks < G / 16; ++ks) {          // 16 channels (32 bytes) per instruction
+                const uint32_t off = (uint32_t)(b * 2 * G + ks * 32) >> 4;
+                mma_bf16(d + b * G, adesc + off, bdesc + off, idesc, (sp | ks) != 0);
+              }
             }
           }
         }
@@ -401,41 +434,50 @@ static TcEncodeFn tc_encode_fn() {
   return fn;
 }
 
-template <int G, bool AMAX>
+template <int G, bool AMAX, int NSPLIT>
 static cudaError_t tc_launch(const CUtensorMap& map, const void* T, int64_t M, int64_t K, const float* ts, uint8_t* codes,
                              uint8_t* scales, int sf, int num_panels, int n_items, int grid, int32_t* status, int cs, bool pdl,
                              const uint32_t* amax_in, float* ts_out, int mx_ceil, int drop, cudaStream_t st) {
-  const __nv_bfloat16* Tb = reinterpret_cast<const __nv_bfloat16*>(T);
+  static bool attr_done_of[kDeviceSlots] = {};           // per instantiation and device
+  const int slot = device_slot();
+  if (slot < 0) return cudaErrorInvalidDevice;
+  constexpr int SMEM = tc::smem_bytes(NSPLIT);
+  if (!attr_done_of[slot]) {
+    const cudaError_t e = cudaFuncSetAttribute(tc::tq_tc_kernel<G, AMAX, NSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    if (e != cudaSuccess) return e;
+    attr_done_of[slot] = true;
+  }
   if (!pdl) {
-    tc::tq_tc_kernel<G, AMAX><<<grid, tc::THREADS, tc::SMEM, st>>>(map, Tb, M, K, ts, codes, scales, sf, num_panels, n_items, status, cs,
-                                                                  amax_in, ts_out, mx_ceil, drop);
+    tc::tq_tc_kernel<G, AMAX, NSPLIT><<<grid, tc::THREADS, SMEM, st>>>(map, T, M, K, ts, codes, scales, sf, num_panels, n_items, status, cs,
+                                                                        amax_in, ts_out, mx_ceil, drop);
     return cudaGetLastError();
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
   cfg.blockDim = dim3(tc::THREADS, 1, 1);
-  cfg.dynamicSmemBytes = tc::SMEM;
+  cfg.dynamicSmemBytes = SMEM;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tc::tq_tc_kernel<G, AMAX>, map, Tb, M, K, ts, codes, scales, sf, num_panels, n_items, status, cs,
+  return cudaLaunchKernelEx(&cfg, tc::tq_tc_kernel<G, AMAX, NSPLIT>, map, T, M, K, ts, codes, scales, sf, num_panels, n_items, status, cs,
                             amax_in, ts_out, mx_ceil, drop);
 }
 
-// Activation side on the tcgen05 kernel.  cudaErrorNotSupported: the caller uses the warp-level streaming kernel.
-cudaError_t run_quantize_act_tc(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts, uint8_t* codes,
-                                uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl, cudaStream_t st,
-                                const QuantOpts& opt) {
+// Common host part: tensor map over the bf16 rows, grid size, dispatch.  NSPLIT = 1: T is bf16 (activation side);
+// NSPLIT = 3: T is the fp32 weight-side transform.  cudaErrorNotSupported: the caller uses the warp-level kernel.
+template <int NSPLIT>
+static cudaError_t tc_run(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts, uint8_t* codes,
+                          uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl, cudaStream_t st,
+                          const QuantOpts& opt) {
   TcEncodeFn enc = tc_encode_fn();
   if (!enc) return cudaErrorNotSupported;
   if ((reinterpret_cast<uintptr_t>(codes) & 31u) != 0) return cudaErrorNotSupported;   // 256-bit code stores
   const int slot = device_slot();
   if (slot < 0) return cudaErrorInvalidDevice;
   static int sm_count_of[kDeviceSlots] = {};
-  static bool attr_done_of[kDeviceSlots] = {};
   cudaError_t e;
   if (sm_count_of[slot] == 0) {
     int sms = 0, major = 0;
@@ -443,12 +485,6 @@ cudaError_t run_quantize_act_tc(const void* X, int64_t M, int64_t K, const void*
     if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, slot)) != cudaSuccess) return e;
     if (major != 10) return cudaErrorNotSupported;
     sm_count_of[slot] = sms;
-  }
-  if (!attr_done_of[slot]) {
-    if ((e = cudaFuncSetAttribute(tc::tq_tc_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(tc::tq_tc_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(tc::tq_tc_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM)) != cudaSuccess) return e;
-    attr_done_of[slot] = true;
   }
   CUtensorMap map;
   const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
@@ -465,27 +501,41 @@ cudaError_t run_quantize_act_tc(const void* X, int64_t M, int64_t K, const void*
   if (items > 0x7fffffff) return cudaErrorNotSupported;
   // CTA c takes items c, c + grid, c + 2 grid, ... and item n of a CTA uses ring stage n % STAGES, so a stage sees
   // the panels (c + grid * n) % panels for n = s, s + STAGES, ...: always the same panel when panels divides
-  // STAGES * grid.  The grid is the largest such number of CTAs (where that keeps at least 3/4 of the SMs busy): a
-  // stage's transforms are then written once per launch.
+  // STAGES * grid.  Preferred: a multiple of the panel count (one panel per CTA); else the largest grid with that
+  // property; each only where it keeps at least 3/4 of the SMs busy.  A stage's transforms are then written once.
   const int sms = sm_count_of[slot];
   int g4 = tc::STAGES, pp = num_panels;                         // gcd(panels, STAGES)
   while (pp != 0) { const int t = g4 % pp; g4 = pp; pp = t; }
   const int step = num_panels / g4;
   int grid = sms;
-  if (num_panels <= sms && (sms / num_panels) * num_panels * 4 >= sms * 3) grid = (sms / num_panels) * num_panels;   // one panel per CTA
-  else if (step <= sms && (sms / step) * step * 4 >= sms * 3) grid = (sms / step) * step;                           // one panel per stage
+  if (num_panels <= sms && (sms / num_panels) * num_panels * 4 >= sms * 3) grid = (sms / num_panels) * num_panels;
+  else if (step <= sms && (sms / step) * step * 4 >= sms * 3) grid = (sms / step) * step;
   if (items < grid) grid = (int)items;
   const int cs = clear_status ? 1 : 0;
   if (opt.amax_out != nullptr) {                 // AbsMax pass only (g = 16)
     if (g != 16) return cudaErrorNotSupported;
-    return tc_launch<16, true>(map, T, M, K, nullptr, nullptr, nullptr, sf, num_panels, (int)items, grid, status, cs, pdl, nullptr,
-                               reinterpret_cast<float*>(opt.amax_out), 0, -1, st);
+    return tc_launch<16, true, NSPLIT>(map, T, M, K, nullptr, nullptr, nullptr, sf, num_panels, (int)items, grid, status, cs, pdl,
+                                       nullptr, reinterpret_cast<float*>(opt.amax_out), 0, -1, st);
   }
   if (g == 32)
-    return tc_launch<32, false>(map, T, M, K, ts, codes, scales, sf, num_panels, (int)items, grid, status, cs, pdl, opt.amax_in,
-                                opt.ts_out, opt.mx_ceil ? 1 : 0, opt.drop_item, st);
-  return tc_launch<16, false>(map, T, M, K, ts, codes, scales, sf, num_panels, (int)items, grid, status, cs, pdl, opt.amax_in,
-                              opt.ts_out, 0, opt.drop_item, st);
+    return tc_launch<32, false, NSPLIT>(map, T, M, K, ts, codes, scales, sf, num_panels, (int)items, grid, status, cs, pdl,
+                                        opt.amax_in, opt.ts_out, opt.mx_ceil ? 1 : 0, opt.drop_item, st);
+  return tc_launch<16, false, NSPLIT>(map, T, M, K, ts, codes, scales, sf, num_panels, (int)items, grid, status, cs, pdl,
+                                      opt.amax_in, opt.ts_out, 0, opt.drop_item, st);
+}
+
+// Activation side (bf16 transforms).
+cudaError_t run_quantize_act_tc(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts, uint8_t* codes,
+                                uint8_t* scales, int sf, int32_t* status, bool clear_status, bool pdl, cudaStream_t st,
+                                const QuantOpts& opt) {
+  return tc_run<1>(X, M, K, T, g, ts, codes, scales, sf, status, clear_status, pdl, st, opt);
+}
+
+// Weight side (Algorithm 2, last line): W[N,K] bf16, Tinv fp32 split three ways inside the kernel.  opt carries the
+// AbsMax pass / tensor-scale pointers for NVFP4 exactly as on the activation side.
+cudaError_t run_quantize_weight_tc(const void* W, int64_t N, int64_t K, const float* Tinv, int g, uint8_t* codes,
+                                   uint8_t* scales, int sf, cudaStream_t st, const QuantOpts& opt) {
+  return tc_run<3>(W, N, K, Tinv, g, nullptr, codes, scales, sf, nullptr, false, false, st, opt);
 }
 
 }  // namespace wush

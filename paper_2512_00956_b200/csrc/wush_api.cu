@@ -163,7 +163,7 @@ int wush_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv,
   if (N == 0) return WUSH_OK;
   cudaError_t e = wush::run_quantize_weight(W, N, K, Tinv, g, w_tensor_scale, codes, scales, (int)sf,
                                             reinterpret_cast<uint32_t*>(workspace), (cudaStream_t)stream,
-                                            fmt == WUSH_MXFP4_CEIL);
+                                            fmt == WUSH_MXFP4_CEIL, forced_rows());
   return e == cudaSuccess ? WUSH_OK : cuda_fail(e);
 }
 

@@ -45,6 +45,8 @@ cudaError_t run_quantize_act_stream(const void* X, int64_t M, int64_t K, const v
 cudaError_t run_quantize_act_tc(const void* X, int64_t M, int64_t K, const void* T, int g, const float* ts,
                                 uint8_t* codes, uint8_t* scales, int sf, int32_t* status, bool clear_status,
                                 bool pdl, cudaStream_t st, const QuantOpts& opt = QuantOpts());
+cudaError_t run_quantize_weight_tc(const void* W, int64_t N, int64_t K, const float* Tinv, int g, uint8_t* codes,
+                                   uint8_t* scales, int sf, cudaStream_t st, const QuantOpts& opt);
 // weight side through the streaming kernel (fp32 Tinv, three-way split); cudaErrorNotSupported = use the other kernel
 cudaError_t run_quantize_weight_stream(const void* W, int64_t N, int64_t K, const float* Tinv, int g, uint8_t* codes,
                                        uint8_t* scales, int sf, cudaStream_t st, const QuantOpts& opt);
@@ -52,7 +54,7 @@ cudaError_t run_transform_f32(const void* X, int64_t M, int64_t K, const void* T
                               float* V, cudaStream_t st);
 cudaError_t run_quantize_weight(const void* W, int64_t N, int64_t K, const float* Tinv, int g,
                                 float* ts_out, uint8_t* codes, uint8_t* scales, int sf,
-                                uint32_t* amax_ws, cudaStream_t st, bool mx_ceil = false);
+                                uint32_t* amax_ws, cudaStream_t st, bool mx_ceil = false, int force_rows = 0);
 cudaError_t run_quantize_f32(const float* V, int64_t R, int64_t K, int g, const float* ts,
                              uint8_t* codes, uint8_t* scales, int sf, cudaStream_t st, bool mx_ceil = false);
 

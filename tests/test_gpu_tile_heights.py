@@ -136,3 +136,29 @@ def test_forced_height_whole_layer(rows, fmt):
     Y2, wsp2 = wush.linear(X, dev_bf16(L.T_bits), wq, ws, fmt, tsx, tsw)
     torch.cuda.synchronize()
     assert torch.equal(Y, Y2) and torch.equal(wsp[: M * K // 2], wsp2[: M * K // 2])
+
+
+@pytest.mark.parametrize("rows", [0, 64])
+@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4", "mxfp4_ceil"])
+def test_weight_quantiser_on_both_kernels(rows, fmt):
+    """wush_quantize_weight (fp32 transforms, exact three-way bf16 split) through the tcgen05 kernel (hook 0, the
+    default for more than 256 rows) and through the warp-level kernel (hook 64), ragged row count and a channel tail:
+    both against the oracle, and bit-identical scale bytes between the two."""
+    g = Q.GROUP[fmt]
+    rng = np.random.default_rng(31)
+    N, K = 1237, 1088
+    W_bits = F.f64_to_bf16_bits(0.02 * rng.standard_normal((N, K)) * np.exp(rng.uniform(-1, 1, (1, K))))
+    Tinv = (rng.standard_normal((K // g, g, g)) / np.sqrt(g)).astype(np.float32)
+    wbar = P.transform_blocks(F.bf16_bits_to_f64(W_bits), Tinv.astype(np.float64)).astype(np.float32)
+    ts = Q.nvfp4_tensor_scale(wbar) if fmt == "nvfp4" else None
+    wush.debug_quantiser_rows(rows)
+    for sf in (wush.SF_LINEAR, wush.SF_TILED):
+        codes, scales, ts_g = wush.quantize_weight(dev_bf16(W_bits), dev(Tinv), fmt, sf=sf)
+        torch.cuda.synchronize()
+        sc = scales.cpu().numpy()
+        if sf == wush.SF_TILED:
+            sc = untile(sc, N, K // g)
+        if fmt == "nvfp4":
+            assert abs(float(ts_g[0].item()) - float(ts)) <= 2e-7 * float(ts)
+        stats = compare_quantized(codes.cpu().numpy(), sc, wbar, fmt, ts)
+        assert stats["flipped_codes"] <= stats["guarded_elems"]
