@@ -300,22 +300,36 @@ def timed(fn, sets, steps, min_ms, dev, barrier=None, what="step"):
 
 
 def library_fp4_gemm_ms(wl, steps, dev):
-    """cuBLASLt's block-scaled FP4 GEMM of the same shape through torch._scaled_mm on this workload's own codes
-    and scale bytes - context beside `bf16_gemm`, never on the product path.  None if torch cannot run it."""
+    """cuBLASLt's block-scaled FP4 GEMM of the same shape through torch._scaled_mm - context beside `bf16_gemm`, never
+    on the product path.  NVFP4 workloads: on this workload's own codes and scale bytes.  MXFP4 workloads: torch in
+    this image refuses E8M0-scaled FP4 operands, so the library runs its NVFP4 kernel on the same codes with unit E4M3
+    scale bytes (same shape, same operand bytes plus twice the scale bytes; a timing stand-in, the values mean nothing).
+    Returns (ms, what) or (None, reason)."""
     import torch
     try:
-        sdt = torch.float8_e8m0fnu if wl.g == 32 else torch.float8_e4m3fn
+        if wl.g == 16:
+            xs = [d_["xs"].view(torch.float8_e4m3fn) for d_ in wl.sets]
+            ws = [d_["wsc"].view(torch.float8_e4m3fn) for d_ in wl.sets]
+            what = "torch._scaled_mm (cuBLASLt NVFP4) on this workload's codes and scales"
+        else:
+            nx = wl.wush.scale_bytes(wl.M, wl.K, 16, wl.wush.SF_TILED)
+            nw = wl.wush.scale_bytes(wl.N, wl.K, 16, wl.wush.SF_TILED)
+            xs = [torch.full((nx,), 0x38, dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn) for _ in wl.sets]
+            ws = [torch.full((nw,), 0x38, dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn) for _ in wl.sets]
+            what = ("torch._scaled_mm (cuBLASLt NVFP4) on this workload's MXFP4 codes with unit E4M3 scales: "
+                    "timing stand-in, torch refuses MXFP4 operands")
+        idx = {id(d_): i for i, d_ in enumerate(wl.sets)}
 
         def fn(d_):
+            i = idx[id(d_)]
             torch._scaled_mm(d_["xq"].view(torch.float4_e2m1fn_x2), d_["wq"].view(torch.float4_e2m1fn_x2).t(),
-                             d_["xs"].view(sdt), d_["wsc"].view(sdt), out_dtype=torch.bfloat16)
+                             xs[i], ws[i], out_dtype=torch.bfloat16)
         fn(wl.sets[0])
         torch.cuda.synchronize()
         ms, _, _, _ = timed(fn, wl.sets, steps, MIN_TIMED_MS_SIDE, dev, what="library fp4 gemm")
-        return ms
+        return ms, what
     except Exception as exc:
-        sys.stderr.write(f"[bench] library FP4 GEMM not available: {str(exc)[:200]}\n")
-        return None
+        return None, str(exc).splitlines()[0][:160]
 
 
 def fractions(wl, peaks, step_ms, q_ms, g_ms):
@@ -383,7 +397,7 @@ def run_ours(args):
 
     bf16_ms, _, _, _ = timed(bf16_step, sets, args.steps, MIN_TIMED_MS_SIDE, dev, None, "bf16 gemm")
     del Wb, Yb
-    lib_ms = library_fp4_gemm_ms(wl, args.steps, dev) if rank == 0 else None
+    lib_ms, lib_what = library_fp4_gemm_ms(wl, args.steps, dev) if rank == 0 else (None, "rank 0 only")
 
     # ---- the two offline kernels of the path (Algorithm 2), timed once each for the record
     def once(fn, reps=5):
@@ -562,9 +576,9 @@ def run_ours(args):
             "roofline": roof, "roofline_quant": roof_q,
             "bf16_gemm": {"ms": bf16_ms, "tflops": flops / (bf16_ms * 1e-3) / 1e12, "speedup_linear": bf16_ms / ms_rank,
                           "speedup_gemm_only": bf16_ms / g_ms, "impl": "torch.matmul (cuBLAS)"},
-            "fp4_gemm_library": None if lib_ms is None else
+            "fp4_gemm_library": {"ms": None, "unavailable": lib_what} if lib_ms is None else
             {"ms": lib_ms, "tflops": flops / (lib_ms * 1e-3) / 1e12, "ours_over_library": lib_ms / g_ms,
-             "impl": "torch._scaled_mm (cuBLASLt block-scaled FP4), context only"},
+             "impl": lib_what + "; context only"},
             "e2e": {"value": e2e_rate / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d_bytes,
                     "d2h_bytes_per_step": d2h_bytes, "ms_per_step": e2e_ms_rank},
             "gpu_launches": (3 if wl.dynamic else 2) * args.steps, "kernel_ms": {"transform_quant": q_ms, "gemm_fp4": g_ms},

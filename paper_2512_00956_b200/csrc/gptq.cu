@@ -27,6 +27,7 @@ namespace wush {
 namespace gq {
 
 constexpr int MOM_PARTS = 64;        // CTAs (= partial sums) of the block-moment kernel
+constexpr int GROUP = 8;             // blocks whose updates of the far columns are applied in one pass
 
 // ---------------------------------------------------------------------------------------- preparation
 __global__ void to_f64_kernel(const __nv_bfloat16* __restrict__ W, double* __restrict__ out, int64_t n) {
@@ -313,29 +314,47 @@ block_quant_kernel(double* __restrict__ Wc, int64_t N, int64_t K, int blk, const
   for (int a = 0; a < D; ++a) zrow[a] = z[a];
 }
 
-// Inter-block propagation: Wc[n][k] += sum_c Z[n][c] * L[k][blk*d + c] for every later column k (L[k][j] = V[j][k]).
-// A thread keeps the d values V[blk*d + c][k] of its column in registers and walks 32 rows.
+// Inter-block propagation for columns k in [k_begin, k_end) and the nb blocks blk0 .. blk0 + nb - 1 whose Z is stored
+// (Z of block blk0 + t at Z + t * N * D):
+//   Wc[n][k] <- (..((Wc[n][k] + u_0) + u_1).. + u_{nb-1}),   u_t = sum_c Z_t[n][c] * L[k][(blk0 + t)*d + c],  L[k][j] = V[j][k]
+// - the additions in block order, each u_t summed over c in order, exactly as if every block had updated all later
+// columns right away.  The solver uses it twice: with nb = 1 for the columns of the current group of blocks (the next
+// block needs them at once) and with nb = the group size for everything beyond the group (one pass over the far
+// columns per group instead of one per block).  A thread owns one column and walks 32 rows.
 template <int D>
 __global__ void __launch_bounds__(256)
-propagate_kernel(double* __restrict__ Wc, int64_t N, int64_t K, int blk, const double* __restrict__ V, const double* __restrict__ Z) {
+propagate_kernel(double* __restrict__ Wc, int64_t N, int64_t K, int blk0, int nb, int64_t k_begin, int64_t k_end,
+                 const double* __restrict__ V, const double* __restrict__ Z) {
   __shared__ double zs[32][D];
-  const int64_t k = (int64_t)(blk + 1) * D + (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int64_t k = k_begin + (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t n0 = (int64_t)blockIdx.y * 32;
-  for (int idx = threadIdx.x; idx < 32 * D; idx += 256) {
-    const int64_t n = n0 + idx / D;
-    zs[idx / D][idx % D] = (n < N) ? Z[n * D + idx % D] : 0.0;
-  }
-  __syncthreads();
-  if (k >= K) return;
-  double v[D];
+  const bool live = k < k_end;
+  double w[32];
 #pragma unroll
-  for (int c = 0; c < D; ++c) v[c] = V[((int64_t)blk * D + c) * K + k];
-  for (int r = 0; r < 32 && n0 + r < N; ++r) {
-    double s = 0.0;
+  for (int r = 0; r < 32; ++r) w[r] = (live && n0 + r < N) ? Wc[(n0 + r) * K + k] : 0.0;
+  for (int t = 0; t < nb; ++t) {
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < 32 * D; idx += 256) {
+      const int64_t n = n0 + idx / D;
+      zs[idx / D][idx % D] = (n < N) ? Z[((int64_t)t * N + n) * D + idx % D] : 0.0;
+    }
+    __syncthreads();
+    if (!live) continue;
+    double v[D];
 #pragma unroll
-    for (int c = 0; c < D; ++c) s += zs[r][c] * v[c];
-    Wc[(n0 + r) * K + k] += s;
+    for (int c = 0; c < D; ++c) v[c] = V[((int64_t)(blk0 + t) * D + c) * K + k];
+#pragma unroll
+    for (int r = 0; r < 32; ++r) {
+      double s = 0.0;
+#pragma unroll
+      for (int c = 0; c < D; ++c) s += zs[r][c] * v[c];
+      w[r] += s;
+    }
   }
+  if (!live) return;
+#pragma unroll
+  for (int r = 0; r < 32; ++r)
+    if (n0 + r < N) Wc[(n0 + r) * K + k] = w[r];
 }
 
 // a failed factorisation of the damped Hessian (non-positive pivot) is reported on every block
@@ -348,11 +367,11 @@ __global__ void report_failure_kernel(const int* __restrict__ fail, int32_t* __r
 
 // ---------------------------------------------------------------------------------------- host side
 // workspace: Wc [N][K] | A (Hd, then U) [K][K] | V [K][K] | MX [K/d][d][d] | Z [N][d] | partial [MOM_PARTS][d][d] |
-//            mw [d][d] | lmat [2][d][d] | fail flag
+//            mw [d][d] | lmat [2][d][d] | fail flag          (Z holds the last GROUP blocks' [N][d])
 static inline size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
 size_t gptq_workspace_bytes(int64_t N, int64_t K, int g) {
   const size_t d2 = (size_t)g * g * sizeof(double);
-  return up256((size_t)N * K * 8) + 2 * up256((size_t)K * K * 8) + up256((size_t)K * g * 8) + up256((size_t)N * g * 8) +
+  return up256((size_t)N * K * 8) + 2 * up256((size_t)K * K * 8) + up256((size_t)K * g * 8) + up256((size_t)gq::GROUP * N * g * 8) +
          up256(gq::MOM_PARTS * d2) + up256(d2) + up256(2 * d2) + 256;
 }
 
@@ -368,7 +387,7 @@ static cudaError_t gptq_run(const void* W, int64_t N, int64_t K, const void* Xc,
   double* A = reinterpret_cast<double*>(p); p += up256((size_t)K * K * 8);
   double* V = reinterpret_cast<double*>(p); p += up256((size_t)K * K * 8);
   double* MX = reinterpret_cast<double*>(p); p += up256((size_t)K * D * 8);
-  double* Z = reinterpret_cast<double*>(p); p += up256((size_t)N * D * 8);
+  double* Z = reinterpret_cast<double*>(p); p += up256((size_t)GROUP * N * D * 8);
   double* partial = reinterpret_cast<double*>(p); p += up256(MOM_PARTS * d2);
   double* mw = reinterpret_cast<double*>(p); p += up256(d2);
   double* lmat = reinterpret_cast<double*>(p); p += up256(2 * d2);
@@ -402,16 +421,27 @@ static cudaError_t gptq_run(const void* W, int64_t N, int64_t K, const void* Xc,
                                      Tinv + (size_t)i * D * D, info ? info + i : nullptr, st)) != cudaSuccess) return e;
     block_hessian_kernel<D><<<1, BT_THREADS, 0, st>>>(Tb + (size_t)i * D * D, V, K, i, lmat, Tinv + (size_t)i * D * D, info); GQ_CHECK();
     const unsigned qgrid = (unsigned)((N + 127) / 128);
+    const int t = i % GROUP;                                  // position inside the current group of blocks
+    double* Zi = Z + (size_t)t * N * D;
     if (fmt == kFmtMX)
       block_quant_kernel<D, kFmtMX><<<qgrid, 128, 0, st>>>(Wc, N, K, i, Tb + (size_t)i * D * D, Tinv + (size_t)i * D * D, lmat, ts_w,
-                                                          mx_ceil, codes, scales, sf, K / D, Z);
+                                                          mx_ceil, codes, scales, sf, K / D, Zi);
     else
       block_quant_kernel<D, kFmtNV><<<qgrid, 128, 0, st>>>(Wc, N, K, i, Tb + (size_t)i * D * D, Tinv + (size_t)i * D * D, lmat, ts_w,
-                                                          0, codes, scales, sf, K / D, Z);
+                                                          0, codes, scales, sf, K / D, Zi);
     GQ_CHECK();
-    const int64_t later = K - (int64_t)(i + 1) * D;
-    if (later > 0) {
-      propagate_kernel<D><<<dim3((unsigned)((later + 255) / 256), (unsigned)((N + 31) / 32)), 256, 0, st>>>(Wc, N, K, i, V, Z);
+    // this block's update: at once for the rest of its group, together with the group's other blocks for all columns
+    // beyond the group (same additions in the same order either way)
+    const int group_first = i - t;
+    const int64_t group_end = (int64_t)min(group_first + GROUP, C) * D;
+    const int64_t near_begin = (int64_t)(i + 1) * D;
+    const unsigned ny = (unsigned)((N + 31) / 32);
+    if (near_begin < group_end) {
+      propagate_kernel<D><<<dim3((unsigned)((group_end - near_begin + 255) / 256), ny), 256, 0, st>>>(Wc, N, K, i, 1, near_begin, group_end, V, Zi);
+      GQ_CHECK();
+    }
+    if ((t == GROUP - 1 || i == C - 1) && group_end < K) {
+      propagate_kernel<D><<<dim3((unsigned)((K - group_end + 255) / 256), ny), 256, 0, st>>>(Wc, N, K, group_first, t + 1, group_end, K, V, Z);
       GQ_CHECK();
     }
   }
