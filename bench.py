@@ -548,6 +548,9 @@ def run_ours(args):
                 gg, _, _, _ = timed(w2.gemm_only, w2.sets, k2, MIN_TIMED_MS_SIDE, dev, None, "gemm")
                 e = {"workload": c_.name, "M": m_, "K": c_.K, "N": c_.N, "format": f_, "status": w2.status()}
                 e.update(fractions(w2, peaks, s_ms, qq, gg))
+                if m_ > 128:                                   # the library's FP4 GEMM of the same shape, for context
+                    lm, _ = library_fp4_gemm_ms(w2, k2, dev)
+                    e["library_gemm_us"] = None if lm is None else lm * 1e3
                 others.append(e)
                 w2.release()
                 del w2
