@@ -328,6 +328,10 @@ cudaError_t run_moments_partial_stream(const void* Xc, int64_t B, int64_t K, int
     sm_count = sms;
   }
   int64_t grid = (int64_t)sm_count * MS_CTAS_PER_SM < MS_DESIGN_SMS ? (int64_t)sm_count * MS_CTAS_PER_SM : MS_DESIGN_SMS;
+  // A multiple of the panel count where that keeps at least 3/4 of the slots: every CTA's run is then a stretch of row
+  // blocks of ONE panel, the CTAs of neighbouring panels start at the same rows and walk down together, so whole rows
+  // of X are fetched at about the same time (DRAM pages used in full) instead of 256-byte pieces of unrelated rows.
+  if (panels <= grid && (grid / panels) * panels * 4 >= grid * 3) grid = (grid / panels) * panels;
   if (items < grid) grid = items;
   int64_t need = (grid + panels - 1) / panels + 1;
   if (need > num_rb) need = num_rb;
