@@ -180,3 +180,28 @@ def test_expired_wait_is_reported_and_the_next_call_works():
     torch.cuda.synchronize()
     assert wush.linear_status(wsp, M, K, 32) == 0
     assert rel_fro(Y.cpu().numpy(), L.forward(d["X"])) <= 1e-3
+
+
+@pytest.mark.parametrize("fmt", ["mxfp4", "nvfp4"])
+def test_one_workspace_serves_every_call(fmt):
+    """wush_workspace_bytes(M, N, K, fmt, g): a single buffer of that size is enough for the moments of W and of the
+    calibration tokens, the weight quantiser and the online layer, and the layer's result is the oracle's."""
+    g = 32 if fmt == "mxfp4" else 16
+    M, N, K, B = 300, 520, 1024, 512
+    d, L = _layer(2, fmt, M=M, N=N, K=K, B=B)
+    need = wush.workspace_bytes(M, N, K, fmt)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    W, Xc, X = dev_bf16(d["W"]), dev_bf16(d["Xc"]), dev_bf16(d["X"])
+    mom_w, cnt_w = wush.calib_moments(W, g, workspace=ws)
+    mom_x, cnt_x = wush.calib_moments(Xc, g, workspace=ws)
+    torch.cuda.synchronize()
+    S = P.second_moment_sums(F.bf16_bits_to_f64(d["W"]), g)
+    assert rel_fro(mom_w.cpu().numpy(), S) <= 1e-5 and int(cnt_w[0].item()) == N and int(cnt_x[0].item()) == B
+    codes, scales = wush._alloc_q(N, K, g, wush.SF_TILED, W.device)
+    tsw = torch.zeros(4, dtype=torch.float32, device="cuda") if fmt == "nvfp4" else None
+    wush.quantize_weight(W, dev(L.T_xvsh32), fmt, sf=wush.SF_TILED, out=(codes, scales, tsw, ws))
+    tsx = dev(np.full(4, L.ts_x, dtype=np.float32)) if fmt == "nvfp4" else None
+    Y, _ = wush.linear(X, dev_bf16(L.T_bits), codes, scales, fmt, tsx, tsw, workspace=ws)
+    torch.cuda.synchronize()
+    assert wush.linear_status(ws, M, K, g) == 0
+    assert rel_fro(Y.cpu().numpy(), L.forward(d["X"])) <= 1e-3
