@@ -89,7 +89,8 @@ const char* wush_status_string(int status);
  * (role << 16) | index: role 0x06 / 0x07 / 0x08 = producer / MMA issuer / epilogue of the quantiser (0x04 / 0x05 =
  * producer / consumer of its warp-level variant; index = work item of the CTA),
  * 0x11..0x15 = producer, scale-copy wait, accumulator hand-over, epilogue, operand wait of the GEMM for
- * M > 128, 0x01..0x03 = producer, MMA issuer, epilogue of the GEMM for M <= 128.  The
+ * M > 128 (0x16 = that kernel found its shared-memory window misplaced and did no work),
+ * 0x01..0x03 = producer, MMA issuer, epilogue of the GEMM for M <= 128.  The
  * caller copies the word to the host after synchronising; this helper maps it to WUSH_OK or WUSH_ERR_TIMEOUT. */
 int wush_decode_status(int32_t word);
 /* Text of the last CUDA error this library saw on the calling thread ("" if none). */

@@ -31,7 +31,9 @@ namespace g2 {
 
 constexpr int BM = 256, BN = 256;       // cluster tile
 constexpr int BKB = 128;                // packed-FP4 bytes per row per stage (256 elements)
-constexpr int STAGES = 5;
+// Ring depth: as deep as shared memory allows.  A K slab's operands take about 2 us from request to arrival under load
+// and 0.27-0.37 us to consume, so the ring is what limits the kernel: MXFP4 stages (35 KB) fit six times, NVFP4 (38 KB) five.
+__host__ __device__ constexpr int stages(int fmt) { return fmt == 0 ? 6 : 5; }
 constexpr int A_BYTES = 128 * BKB;      // this CTA's 128 rows of A
 constexpr int B_BYTES = 128 * BKB;      // this CTA's 128 rows (half) of B
 constexpr int EPI_WARPS = 8;
@@ -39,14 +41,19 @@ constexpr int SF_WARP = 2 + EPI_WARPS;     // copies scale tiles to tensor memor
 constexpr int THREADS = (3 + EPI_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
 // scale tiles: one 48-column buffer per ring stage (A scales 16 columns, B scales 32), after the accumulator
-constexpr uint32_t SF_COL0 = 256, SF_STRIDE = 48, SFB_OFF = 16;
+constexpr uint32_t SF_COL0 = 256, SFB_OFF = 16;
+// tensor-memory columns of one stage's scale buffer: A 8 / 16 columns from column 0, B 16 / 32 from column 16
+__host__ __device__ constexpr uint32_t sf_stride(int fmt) { return fmt == 0 ? 32u : 48u; }
 constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;   // clears the CTA-rank bit of a shared::cluster address: rank 0 of the pair
 
 __host__ __device__ constexpr int tps(int fmt) { return fmt == kFmtMX ? 2 : 4; }
 __host__ __device__ constexpr int sf_bytes(int fmt) { return 3 * tps(fmt) * 512; }
 __host__ __device__ constexpr int stage_bytes(int fmt) { return A_BYTES + B_BYTES + sf_bytes(fmt); }
-constexpr int EPI_STAGE_BYTES = 32 * 128;   // per epilogue warp: 32 rows x 128 bytes, 128-byte swizzle
-__host__ __device__ constexpr int smem_bytes(int fmt) { return 1024 + STAGES * stage_bytes(fmt) + EPI_WARPS * EPI_STAGE_BYTES + 256; }
+// rows of one output box: an epilogue warp pushes its 32 rows in two halves where that buys a ring stage (MXFP4)
+__host__ __device__ constexpr int epi_rows(int fmt) { return fmt == 0 ? 16 : 32; }
+__host__ __device__ constexpr int epi_stage_bytes(int fmt) { return epi_rows(fmt) * 128; }   // per epilogue warp, 128-byte swizzle
+// the alignment slack is 768 bytes: the ring must start on a 1 KiB boundary and the dynamic window starts on a 256-byte one
+__host__ __device__ constexpr int smem_bytes(int fmt) { return 768 + stages(fmt) * stage_bytes(fmt) + EPI_WARPS * epi_stage_bytes(fmt) + 256; }
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
@@ -164,6 +171,9 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
                      int M, int N, int K, const float* __restrict__ tsx, const float* __restrict__ tsw,
                      const __grid_constant__ CUtensorMap mapY, int out_bf16, int32_t* __restrict__ status, int clear_status) {
   constexpr int TPS = tps(FMT);
+  constexpr int STAGES = stages(FMT);
+  constexpr uint32_t SF_STRIDE = sf_stride(FMT);
+  constexpr int EPI_ROWS = epi_rows(FMT), EPI_STAGE_BYTES = epi_stage_bytes(FMT);
   constexpr int KSTEPS_PER_TILE = (FMT == kFmtMX) ? 2 : 1;
   extern __shared__ uint8_t raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
@@ -181,6 +191,17 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  {
+    // The window is sized with 768 bytes to spare for the 1 KiB alignment of the ring.  Its start is the same in
+    // every CTA of the grid, so if it ever sat less than 256-byte aligned all CTAs leave here together, before any
+    // barrier or tensor memory exists, and the call reports it.
+    uint32_t dyn;
+    asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+    if (static_cast<uint32_t>(smem - raw) + smem_bytes(FMT) - 768 > dyn) {
+      if (threadIdx.x == 0 && blockIdx.x == 0 && status) atomicExch(status, 0x160000);
+      return;
+    }
+  }
   const uint32_t rank = cluster_rank();            // 0 = leader
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
   const int tiles_n = (N + BN - 1) / BN, tiles_m = (M + BM - 1) / BM;
@@ -397,18 +418,18 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) arrive_leader(s32(tmem_empty));
-      // Store through shared memory and TMA: the warp writes its 32 rows x 128 bytes (swizzled, so the 16-byte
-      // row pieces of the 32 lanes spread over all banks) and one lane hands the box to the TMA unit, which
-      // writes whole 128-byte lines and clips rows >= M and columns >= N by itself.
+      // Store through shared memory and TMA: the warp (for MXFP4 half of it at a time, the buffer being kept at 16
+      // rows so that the operand ring can have one more stage) writes its rows x 128 bytes (swizzled, so the 16-byte
+      // row pieces spread over all banks) and one lane hands the box to the TMA unit, which writes whole 128-byte
+      // lines and clips rows >= M and columns >= N by itself.
       uint8_t* stage = sEpi + (warp - 2) * EPI_STAGE_BYTES;
       const uint32_t stage_u32 = s32(stage);
-      const bool rows_ok = (m0 + q * 32) < M;              // warp-uniform
-      auto push_box = [&](int col) {                      // buffer filled: hand it to the TMA unit
+      auto push_box = [&](int col, int row) {             // buffer filled: hand it to the TMA unit
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) {
           asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                       ::"l"(&mapY), "r"(col), "r"(m0 + q * 32), "r"(stage_u32) : "memory");
+                       ::"l"(&mapY), "r"(col), "r"(row), "r"(stage_u32) : "memory");
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       };
@@ -416,39 +437,52 @@ gemm_fp4_2cta_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_cons
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncwarp();
       };
-      uint8_t* my_row = stage + lane * 128;
+      uint8_t* my_row = stage + (lane & (EPI_ROWS - 1)) * 128;
+      const int my_half = lane / EPI_ROWS;
       if (out_bf16) {
 #pragma unroll
         for (int sub = 0; sub < 2; ++sub) {                 // 64 columns (128 bytes of bf16) per box
           const int col = n0 + sub * 64;
-          if (rows_ok && col < N) {
+          if (col >= N) continue;                           // warp-uniform
+#pragma unroll
+          for (int h = 0; h < 32 / EPI_ROWS; ++h) {
+            const int row = m0 + q * 32 + h * EPI_ROWS;
+            if (row >= M) break;                            // warp-uniform
             buffer_free();
+            if (my_half == h) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {                   // chunk j = columns 8j..8j+7 = r[2*sub + j/4][8*(j%4)..]
-              uint32_t p[4];
+              for (int j = 0; j < 8; ++j) {                 // chunk j = columns 8j..8j+7 = r[2*sub + j/4][8*(j%4)..]
+                uint32_t p[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * sub + (j >> 2)][8 * (j & 3) + 2 * e]) * alpha,
-                                                         __uint_as_float(r[2 * sub + (j >> 2)][8 * (j & 3) + 2 * e + 1]) * alpha);
-                p[e] = *reinterpret_cast<uint32_t*>(&h);
+                for (int e = 0; e < 4; ++e) {
+                  __nv_bfloat162 v = __floats2bfloat162_rn(__uint_as_float(r[2 * sub + (j >> 2)][8 * (j & 3) + 2 * e]) * alpha,
+                                                           __uint_as_float(r[2 * sub + (j >> 2)][8 * (j & 3) + 2 * e + 1]) * alpha);
+                  p[e] = *reinterpret_cast<uint32_t*>(&v);
+                }
+                *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
               }
-              *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) = make_uint4(p[0], p[1], p[2], p[3]);
             }
-            push_box(col);
+            push_box(col, row);
           }
         }
       } else {
 #pragma unroll
         for (int sub = 0; sub < 4; ++sub) {                 // 32 columns (128 bytes of fp32) per box
           const int col = n0 + sub * 32;
-          if (rows_ok && col < N) {
-            buffer_free();
+          if (col >= N) continue;                           // warp-uniform
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) =
-                  make_uint4(__float_as_uint(__uint_as_float(r[sub][4 * j]) * alpha), __float_as_uint(__uint_as_float(r[sub][4 * j + 1]) * alpha),
-                             __float_as_uint(__uint_as_float(r[sub][4 * j + 2]) * alpha), __float_as_uint(__uint_as_float(r[sub][4 * j + 3]) * alpha));
-            push_box(col);
+          for (int h = 0; h < 32 / EPI_ROWS; ++h) {
+            const int row = m0 + q * 32 + h * EPI_ROWS;
+            if (row >= M) break;                            // warp-uniform
+            buffer_free();
+            if (my_half == h) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(my_row + ((j ^ (lane & 7)) << 4)) =
+                    make_uint4(__float_as_uint(__uint_as_float(r[sub][4 * j]) * alpha), __float_as_uint(__uint_as_float(r[sub][4 * j + 1]) * alpha),
+                               __float_as_uint(__uint_as_float(r[sub][4 * j + 2]) * alpha), __float_as_uint(__uint_as_float(r[sub][4 * j + 3]) * alpha));
+            }
+            push_box(col, row);
           }
         }
       }
@@ -505,11 +539,11 @@ static bool map_scales(CUtensorMap* map, const void* base, int64_t total_tiles, 
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// output [M][N] bf16 or fp32; box = 128 bytes x 32 rows, 128-byte swizzle
-static bool map_output(CUtensorMap* map, void* Y, int64_t M, int64_t N, int out_bf16) {
+// output [M][N] bf16 or fp32; box = 128 bytes x 16 (MXFP4) or 32 (NVFP4) rows, 128-byte swizzle
+static bool map_output(CUtensorMap* map, void* Y, int64_t M, int64_t N, int out_bf16, int fmt) {
   const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
   const cuuint64_t strides[1] = {(cuuint64_t)N * (out_bf16 ? 2 : 4)};
-  const cuuint32_t box[2] = {(cuuint32_t)(out_bf16 ? 64 : 32), 32};
+  const cuuint32_t box[2] = {(cuuint32_t)(out_bf16 ? 64 : 32), (cuuint32_t)g2::epi_rows(fmt)};
   const cuuint32_t estr[2] = {1, 1};
   return enc_fn()(map, out_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, Y, dims, strides,
                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -582,7 +616,7 @@ cudaError_t run_gemm_fp4_2cta(const uint8_t* Xq, const uint8_t* Xs, const uint8_
   if (!enc_fn()) return cudaErrorNotSupported;
   const int64_t ktiles = ((K / (fmt == kFmtMX ? 32 : 16)) + 3) / 4;
   CUtensorMap a, b, sa, sb, y;
-  if (!map_output(&y, Y, M, N, out_bf16) || !map_bytes(&a, Xq, M, K / 2, 128) || !map_bytes(&b, Wq, N, K / 2, 128) ||
+  if (!map_output(&y, Y, M, N, out_bf16, fmt) || !map_bytes(&a, Xq, M, K / 2, 128) || !map_bytes(&b, Wq, N, K / 2, 128) ||
       !map_scales(&sa, Xs, ((M + 127) / 128) * ktiles, g2::tps(fmt)) ||
       !map_scales(&sb, Ws, ((N + 127) / 128) * ktiles, g2::tps(fmt)))
     return cudaErrorNotSupported;
