@@ -8,7 +8,7 @@
 // N/128 CTAs keep every SM pulling weight bytes.  (M > 128 goes to the two-CTA kernel.)
 // Warp 0 streams operands: per 256-element K slab two TMA tile loads (128-byte swizzle, K-major
 // packed FP4 bytes) and the matching scale tiles (plain bulk copies of the 512-byte GEMM-native
-// scale tiles) into a 3-stage ring guarded by full/empty mbarriers.  One thread of warp 1 copies the scale tiles into tensor memory
+// scale tiles) into a ring of 3 to 5 stages (see stages_of) guarded by full/empty mbarriers.  One thread of warp 1 copies the scale tiles into tensor memory
 // (tcgen05.cp) and issues four K=64 MMAs per slab; tcgen05.commit releases the stage.
 // Warps 2-5 drain the accumulator (tcgen05.ld), apply alpha and store Y.
 //
@@ -26,8 +26,7 @@ namespace wush {
 constexpr int BM = 128;             // tile rows (tokens)
 constexpr int BN = 128;             // tile columns (output channels)
 constexpr int BKB = 128;            // bytes of packed FP4 per row per stage = 256 elements
-constexpr int STAGES = 3;           // two CTAs share an SM: six stages in flight per SM
-constexpr int A_BYTES = BM * BKB;   // 16 KiB
+constexpr int A_BYTES = BM * BKB;   // 16 KiB: what one MMA reads, whatever part of it the A box fills
 constexpr int B_BYTES = BN * BKB;   // 16 KiB
 constexpr int GEMM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 256;  // two co-resident CTAs fit in the 512 columns of an SM
@@ -36,9 +35,20 @@ constexpr uint32_t SFB_COL = 160;   // B scales: 4 columns per scale tile
 
 __host__ __device__ constexpr int sf_tiles_per_stage(int fmt) { return fmt == kFmtMX ? 2 : 4; }
 __host__ __device__ constexpr int stage_sf_bytes(int fmt) { return 2 * sf_tiles_per_stage(fmt) * 512; }
-__host__ __device__ constexpr int gemm_smem_bytes(int fmt) {
-  return 1024 /*alignment slack*/ + STAGES * (A_BYTES + B_BYTES + stage_sf_bytes(fmt)) + 256 /*barriers*/;
+// Ring depth.  The kernel is bound by streaming the weights, and what a CTA streams is set by the bytes it has in
+// flight (about 2 us from request to arrival under load): with few tokens the activation slot of a stage shrinks
+// to the rows that exist (a_rows = 16, 32, 64 or 128) and the ring gets as many stages as still let two CTAs share
+// an SM (3 with 128 rows; 5 with 16).  An MMA always reads 128 rows: the rows beyond the slot are whatever follows
+// it in the ring (all FP4 bit patterns are finite numbers) and only reach accumulator rows that are never stored.
+constexpr int SMEM_PER_CTA = (228 * 1024 - 2 * 1024) / 2;   // two CTAs per SM, 1 KiB reserved for each
+__host__ __device__ constexpr int stage_bytes(int fmt, int a_rows) { return a_rows * BKB + B_BYTES + stage_sf_bytes(fmt); }
+__host__ __device__ constexpr int stages_of(int fmt, int a_rows) { return (SMEM_PER_CTA - 1024 - 256) / stage_bytes(fmt, a_rows); }
+__host__ __device__ constexpr int gemm_smem_bytes(int fmt, int a_rows) {
+  // alignment slack + ring + barriers; the last activation slot is read 16 KiB deep, so with short slots the
+  // weight slots that follow it must exist: they do, the ring is laid out [A slots][B slots][scale tiles]
+  return 1024 + stages_of(fmt, a_rows) * stage_bytes(fmt, a_rows) + 256;
 }
+static_assert(stages_of(kFmtMX, 128) == 3 && stages_of(kFmtNV, 128) == 3 && stages_of(kFmtMX, 16) == 5 && stages_of(kFmtNV, 16) == 5, "ring depth");
 
 // ------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -157,7 +167,7 @@ __device__ __forceinline__ uint32_t instr_desc(int fmt, uint32_t sf_byte) {
 }
 
 // ------------------------------------------------------------------------------ the kernel
-template <int FMT>
+template <int FMT, int A_ROWS>
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const uint8_t* __restrict__ SFA, const uint8_t* __restrict__ SFB, int M, int N, int K,
@@ -165,10 +175,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 int out_bf16, int32_t* __restrict__ status, int a_box_bytes, int clear_status) {
   constexpr int TPS = sf_tiles_per_stage(FMT);           // scale tiles (4 scale columns each) per stage
   constexpr int KSTEPS_PER_TILE = (FMT == kFmtMX) ? 2 : 1;  // K=64 MMAs covered by one scale tile
+  constexpr int STAGES = stages_of(FMT, A_ROWS);
+  constexpr int A_SLOT = A_ROWS * BKB;                   // bytes between the activation slots of consecutive stages
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
-  uint8_t* sB = sA + STAGES * A_BYTES;
+  uint8_t* sB = sA + STAGES * A_SLOT;
   uint8_t* sSF = sB + STAGES * B_BYTES;                   // per stage: [A tiles][B tiles]
   uint64_t* bars = reinterpret_cast<uint64_t*>(sSF + STAGES * stage_sf_bytes(FMT));
   uint64_t* full_bar = bars;
@@ -224,7 +236,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       // the A box covers only round_up(M, 8) rows when M < 128: the rows of the stage below it keep stale
       // bytes, which only reach accumulator rows that are never stored
       uint8_t* sf = sSF + s * stage_sf_bytes(FMT);
-      tma_load_2d(smem_u32(sA + s * A_BYTES), &mapA, kb * BKB, m0, bar);
+      tma_load_2d(smem_u32(sA + s * A_SLOT), &mapA, kb * BKB, m0, bar);
       bulk_load_1d(smem_u32(sf), SFA + ((int64_t)(m0 >> 7) * ktiles_total + kb * TPS) * 512, sf_bytes, bar);
     };
     if (elect_one())
@@ -283,7 +295,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
       const int tiles = min(TPS, ktiles_total - kb * TPS);
       const uint32_t sf = smem_u32(sSF + s * stage_sf_bytes(FMT));
       const int ksteps = min(4, (K - kb * 2 * BKB) / 64);
-      const uint64_t adesc = operand_desc(smem_u32(sA + s * A_BYTES));
+      const uint64_t adesc = operand_desc(smem_u32(sA + s * A_SLOT));
       const uint64_t bdesc = operand_desc(smem_u32(sB + s * B_BYTES));
       if (elect_one()) {
         for (int i = 0; i < tiles; ++i) {
@@ -427,26 +439,27 @@ cudaError_t run_gemm_fp4(const uint8_t* Xq, const uint8_t* Xs, const uint8_t* Wq
   cfg.attrs = attr;
   cfg.numAttrs = after_quantizer ? 1 : 0;          // programmatic dependent of the quantiser inside wush_linear
   const int mi = (int)M, ni = (int)N, ki = (int)K, a_bytes = a_rows * BKB;
-  const int slot = device_slot();
-  if (slot < 0) return cudaErrorInvalidDevice;
-  if (fmt == kFmtMX) {
-    static bool attr_done[kDeviceSlots] = {};
+  const int slot_rows = a_rows <= 16 ? 16 : a_rows <= 32 ? 32 : a_rows <= 64 ? 64 : 128;
+  auto go = [&](auto kernel, int smem, bool* attr_done) -> cudaError_t {
+    const int slot = device_slot();
+    if (slot < 0) return cudaErrorInvalidDevice;
     if (!attr_done[slot]) {
-      e = cudaFuncSetAttribute(gemm_fp4_kernel<kFmtMX>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(kFmtMX));
-      if (e != cudaSuccess) return e;
+      const cudaError_t ea = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      if (ea != cudaSuccess) return ea;
       attr_done[slot] = true;
     }
-    cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtMX);
-    return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtMX>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes, cs);
+    cfg.dynamicSmemBytes = smem;
+    return cudaLaunchKernelEx(&cfg, kernel, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes, cs);
+  };
+#define WUSH_GEMM_CASE(F, R)                                                                  \
+  if (fmt == F && slot_rows == R) {                                                           \
+    static bool attr_done[kDeviceSlots] = {};                                                 \
+    return go(gemm_fp4_kernel<F, R>, gemm_smem_bytes(F, R), attr_done);                       \
   }
-  static bool attr_done[kDeviceSlots] = {};
-  if (!attr_done[slot]) {
-    e = cudaFuncSetAttribute(gemm_fp4_kernel<kFmtNV>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(kFmtNV));
-    if (e != cudaSuccess) return e;
-    attr_done[slot] = true;
-  }
-  cfg.dynamicSmemBytes = gemm_smem_bytes(kFmtNV);
-  return cudaLaunchKernelEx(&cfg, gemm_fp4_kernel<kFmtNV>, mapA, mapB, Xs, Ws, mi, ni, ki, tsx, tsw, Y, out_bf16, status, a_bytes, cs);
+  WUSH_GEMM_CASE(kFmtMX, 16) WUSH_GEMM_CASE(kFmtMX, 32) WUSH_GEMM_CASE(kFmtMX, 64) WUSH_GEMM_CASE(kFmtMX, 128)
+  WUSH_GEMM_CASE(kFmtNV, 16) WUSH_GEMM_CASE(kFmtNV, 32) WUSH_GEMM_CASE(kFmtNV, 64) WUSH_GEMM_CASE(kFmtNV, 128)
+#undef WUSH_GEMM_CASE
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace wush
