@@ -526,7 +526,7 @@ def run_ours(args):
     if world == 1 and not args.no_workloads:
         shared = (wl.W, wl.Xc) if cfg.index == 5 else (None, None)
         wl.release()
-        plan = [(5, "mxfp4", 4096), (5, "nvfp4", 4096), (5, "mxfp4", 128), (5, "mxfp4", 1), (3, "mxfp4", None),
+        plan = [(5, "mxfp4", 4096), (5, "nvfp4", 4096), (5, "mxfp4", 1024), (5, "mxfp4", 128), (5, "mxfp4", 16), (5, "mxfp4", 1), (3, "mxfp4", None),
                 (4, "mxfp4", None), (4, "nvfp4", None), (2, "nvfp4", None)]
         cache = {5: shared}
         for ci, f_, m_ in plan:
