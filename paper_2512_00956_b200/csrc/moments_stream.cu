@@ -73,6 +73,7 @@ __device__ __forceinline__ uint4 ms_ldmatrix_x4_trans(uint32_t addr) {
 }
 
 // the CTA (of `grid`) whose contiguous run [floor(c I / grid), floor((c+1) I / grid)) holds item `it`
+constexpr int MS_FOLD = 32;     // tiles between two folds of the tensor-core sums into the rounded totals
 __host__ __device__ __forceinline__ int ms_cta_of_item(int64_t it, int64_t items, int grid) {
   return static_cast<int>(((it + 1) * grid - 1) / items);
 }
@@ -153,9 +154,16 @@ moments_stream_kernel(const __grid_constant__ CUtensorMap mapX, int64_t K, float
     const uint32_t cbase = 4 * (sbi & 1);     // first chunk of the super-block in its box row
     const uint32_t swz = lane & 7;            // (row & 7) of every row this lane addresses
     constexpr int NT = (G == 32) ? 8 : 4;     // accumulator tiles (16 x 8): g=32: [mt][nt], g=16: [block][nt]
-    float acc[NT][4];
+    // Two levels of fp32 sums.  The tensor core adds into `acc` with truncation, a bias of up to one unit in the
+    // last place of the running sum per MMA; over the ~10^3 tiles of a CTA's run that reached 1e-4 of a diagonal
+    // sum at 2.6e5 tokens.  Every MS_FOLD tiles `acc` is added to `tot` with a rounded fp32 addition and cleared,
+    // so the biased sums stay short.
+    float acc[NT][4], tot[NT][4];
 #pragma unroll
-    for (int a = 0; a < NT; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
+    for (int a = 0; a < NT; ++a) {
+      acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
+      tot[a][0] = tot[a][1] = tot[a][2] = tot[a][3] = 0.f;
+    }
 
     const int64_t seg_stride = K * G;         // floats of one segment of partial sums
     auto flush = [&](int panel) {
@@ -164,7 +172,7 @@ moments_stream_kernel(const __grid_constant__ CUtensorMap mapX, int64_t K, float
 #pragma unroll
       for (int a = 0; a < NT; ++a)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) mine[(a * 4 + e) * 32] = acc[a][e];
+        for (int e = 0; e < 4; ++e) mine[(a * 4 + e) * 32] = __fadd_rn(tot[a][e], acc[a][e]);
       asm volatile("bar.sync 1, %0;" ::"n"(MS_CONSUMERS * 32) : "memory");
       const int sb = panel * MS_PANEL_SB + sbi;
       if (tq == 0 && sb < total_sb) {
@@ -196,7 +204,10 @@ moments_stream_kernel(const __grid_constant__ CUtensorMap mapX, int64_t K, float
       }
       asm volatile("bar.sync 1, %0;" ::"n"(MS_CONSUMERS * 32) : "memory");   // the buffer may be rewritten
 #pragma unroll
-      for (int a = 0; a < NT; ++a) acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
+      for (int a = 0; a < NT; ++a) {
+        acc[a][0] = acc[a][1] = acc[a][2] = acc[a][3] = 0.f;
+        tot[a][0] = tot[a][1] = tot[a][2] = tot[a][3] = 0.f;
+      }
     };
 
     int n = 0;
@@ -248,6 +259,12 @@ moments_stream_kernel(const __grid_constant__ CUtensorMap mapX, int64_t K, float
       }
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ms_u32(&empty_bar[s])) : "memory");
+      if ((n % MS_FOLD) == MS_FOLD - 1) {
+#pragma unroll
+        for (int a = 0; a < NT; ++a)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { tot[a][e] = __fadd_rn(tot[a][e], acc[a][e]); acc[a][e] = 0.f; }
+      }
       if (++rb == num_rb) { rb = 0; ++panel; }
     }
     if (item_end > item_begin) flush(cur_panel);

@@ -27,8 +27,8 @@ def dev(a):
 
 
 def tiled_offsets(rows, KB):
-    """Byte offset of scale (r, kb) in the GEMM-native layout, for all r, kb."""
-    r = np.arange(rows)[:, None]
+    """Byte offset of scale (r, kb) in the GEMM-native layout, for all kb and all r < rows (or the rows listed)."""
+    r = (np.arange(rows) if np.isscalar(rows) else np.asarray(rows, dtype=np.int64))[:, None]
     kb = np.arange(KB)[None, :]
     ktiles = (KB + 3) // 4
     return ((r // 128) * ktiles + kb // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4
