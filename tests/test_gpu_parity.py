@@ -154,7 +154,10 @@ def test_calib_moments(g, B, K):
 # ------------------------------------------------------------------ GEMM alone (oracle's codes in)
 @pytest.mark.parametrize("fmt,M,N,K", [
     ("mxfp4", 128, 256, 256), ("mxfp4", 3, 8, 64), ("mxfp4", 200, 264, 448), ("mxfp4", 128, 2048, 2048),
-    ("nvfp4", 128, 256, 256), ("nvfp4", 5, 16, 64), ("nvfp4", 131, 392, 320), ("nvfp4", 300, 1024, 1536)])
+    ("nvfp4", 128, 256, 256), ("nvfp4", 5, 16, 64), ("nvfp4", 131, 392, 320), ("nvfp4", 300, 1024, 1536),
+    # every activation-slot height of the M <= 128 kernel (16, 32, 64 rows), K long enough for its ring to wrap
+    ("mxfp4", 9, 264, 2560), ("nvfp4", 16, 128, 2304), ("mxfp4", 24, 136, 2048), ("nvfp4", 32, 264, 2048),
+    ("mxfp4", 50, 128, 1792), ("nvfp4", 64, 136, 2048), ("nvfp4", 33, 8, 1536), ("mxfp4", 100, 72, 1600)])
 def test_gemm_fp4_against_oracle_product(fmt, M, N, K):
     d, L = _layer(1, fmt, M=M, N=N, K=K, B=256)
     g = G[fmt]
