@@ -109,15 +109,14 @@ __device__ __forceinline__ void ld32(uint32_t taddr, uint32_t (&u)[32]) {
 template <int G>
 __device__ __forceinline__ uint32_t quantise_block(const uint32_t* u, int mx_ceil, const NvScaleFast& nvf, uint32_t nv_mult_u32,
                                                    uint32_t* words) {
-  float v[G];
-#pragma unroll
-  for (int i = 0; i < G; ++i) v[i] = __uint_as_float(u[i]);
-  // AbsMax as two chains of 3-input maxima (sm_100 has a 3-input FMNMX)
-  float a0 = fmaxf(fabsf(v[0]), fabsf(v[1])), a1 = fmaxf(fabsf(v[2]), fabsf(v[3]));
+  // the values are used where tcgen05.ld left them (no copies): AbsMax as two chains of 3-input maxima (sm_100 has a
+  // 3-input FMNMX), then packed multiplies into fresh registers that feed the conversions
+  auto f = [&](int i) { return __uint_as_float(u[i]); };
+  float a0 = fmaxf(fabsf(f(0)), fabsf(f(1))), a1 = fmaxf(fabsf(f(2)), fabsf(f(3)));
 #pragma unroll
   for (int i = 4; i < G; i += 4) {
-    a0 = fmaxf(fmaxf(a0, fabsf(v[i])), fabsf(v[i + 1]));
-    a1 = fmaxf(fmaxf(a1, fabsf(v[i + 2])), fabsf(v[i + 3]));
+    a0 = fmaxf(fmaxf(a0, fabsf(f(i))), fabsf(f(i + 1)));
+    a1 = fmaxf(fmaxf(a1, fabsf(f(i + 2))), fabsf(f(i + 3)));
   }
   const float a = fmaxf(a0, a1);
   uint32_t byte;
@@ -130,11 +129,11 @@ __device__ __forceinline__ uint32_t quantise_block(const uint32_t* u, int mx_cei
   }
   const uint64_t mm = pair_of(mult);
 #pragma unroll
-  for (int i = 0; i < G; i += 2) mul2_rn(v[i], v[i + 1], mm);
-#pragma unroll
   for (int w = 0; w < G / 8; ++w) {
-    const float (&v8)[8] = *reinterpret_cast<const float (*)[8]>(&v[8 * w]);
-    words[w] = pack_e2m1x8_fast(v8);
+    float p[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) mul2_rn_to(p[2 * i], p[2 * i + 1], f(8 * w + 2 * i), f(8 * w + 2 * i + 1), mm);
+    words[w] = pack_e2m1x8_fast(p);
   }
   return byte;
 }
@@ -501,15 +500,17 @@ static cudaError_t tc_run(const void* X, int64_t M, int64_t K, const void* T, in
   if (items > 0x7fffffff) return cudaErrorNotSupported;
   // CTA c takes items c, c + grid, c + 2 grid, ... and item n of a CTA uses ring stage n % STAGES, so a stage sees
   // the panels (c + grid * n) % panels for n = s, s + STAGES, ...: always the same panel when panels divides
-  // STAGES * grid.  Preferred: a multiple of the panel count (one panel per CTA); else the largest grid with that
-  // property; each only where it keeps at least 3/4 of the SMs busy.  A stage's transforms are then written once.
+  // STAGES * grid, and a stage's transforms are then written once.  The grid is the largest with that property (a
+  // multiple of panels / gcd(panels, STAGES): 144 CTAs for K = 8192, 140 for K = 14336), provided it keeps at least
+  // 3/4 of the SMs busy.  With the GPU to itself the kernel is bound by HBM and a multiple of the panel count (128,
+  // 112 CTAs) is as fast; behind FP4 GEMMs, with the SM clock held down by the power cap, it is bound by the SMs and
+  // the larger grid is 9-12 % faster (16384 x 8192: 72.8 -> 66.2 us).
   const int sms = sm_count_of[slot];
   int g4 = tc::STAGES, pp = num_panels;                         // gcd(panels, STAGES)
   while (pp != 0) { const int t = g4 % pp; g4 = pp; pp = t; }
   const int step = num_panels / g4;
   int grid = sms;
-  if (num_panels <= sms && (sms / num_panels) * num_panels * 4 >= sms * 3) grid = (sms / num_panels) * num_panels;
-  else if (step <= sms && (sms / step) * step * 4 >= sms * 3) grid = (sms / step) * step;
+  if (step <= sms && (sms / step) * step * 4 >= sms * 3) grid = (sms / step) * step;
   if (items < grid) grid = (int)items;
   const int cs = clear_status ? 1 : 0;
   if (opt.amax_out != nullptr) {                 // AbsMax pass only (g = 16)

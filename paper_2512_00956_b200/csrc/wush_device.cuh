@@ -66,6 +66,15 @@ __device__ __forceinline__ void mul2_rn(float& a, float& b, uint64_t mm) {
       : "+f"(a), "+f"(b)
       : "l"(mm));
 }
+// (x, y) = (a, b) * (m, m), results in registers of their own
+__device__ __forceinline__ void mul2_rn_to(float& x, float& y, float a, float b, uint64_t mm) {
+  asm("{\n\t.reg .b64 v;\n\t"
+      "mov.b64 v, {%2, %3};\n\t"
+      "mul.rn.f32x2 v, v, %4;\n\t"
+      "mov.b64 {%0, %1}, v;\n\t}"
+      : "=f"(x), "=f"(y)
+      : "f"(a), "f"(b), "l"(mm));
+}
 // (a, b) * (m, m) with one packed fp32 instruction (round to nearest, no flush)
 __device__ __forceinline__ void mul2_rn(float& a, float& b, float m) {
   asm("{\n\t.reg .b64 v, s;\n\t"
