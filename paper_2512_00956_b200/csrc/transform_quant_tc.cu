@@ -497,7 +497,7 @@ static cudaError_t tc_run(const void* X, int64_t M, int64_t K, const void* T, in
   const int num_rb = (int)((M + tc::ROWS - 1) / tc::ROWS);
   const int num_panels = (int)((K / 64 + tc::SUBS - 1) / tc::SUBS);
   const int64_t items = (int64_t)num_panels * num_rb;
-  if (items > 0x7fffffff) return cudaErrorNotSupported;
+  if (items > 0x70000000) return cudaErrorNotSupported;       // item indices are ints and are stepped past the end by up to two grids
   // CTA c takes items c, c + grid, c + 2 grid, ... and item n of a CTA uses ring stage n % STAGES, so a stage sees
   // the panels (c + grid * n) % panels for n = s, s + STAGES, ...: always the same panel when panels divides
   // STAGES * grid, and a stage's transforms are then written once.  The grid is the largest with that property (a
