@@ -141,16 +141,28 @@ __global__ void __launch_bounds__(256) ul_store_pivot_kernel(double* __restrict_
 
 // One row of V = U^-1 (upper triangular), rows taken from the last to the first:
 //   V[i][i] = 1 / U[i][i],   V[i][c] = -(sum_{k = i+1..c} U[i][k] V[k][c]) / U[i][i]   for c > i.
-// One thread per column c; V[k][c] is read along rows, U[i][k] is the same for the whole warp.
-__global__ void __launch_bounds__(256) uinv_row_kernel(const double* __restrict__ U, double* __restrict__ V, int64_t K, int i) {
-  const int64_t c = (int64_t)i + (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (c >= K) return;
+// A CTA takes 32 columns (lane = column, so V[k][c] is read along rows); its 16 warps take the terms k = i+1+w,
+// i+1+w+16, ... and the 16 partial sums are added in warp order, so the result is the same from run to run.
+// (One thread per column walking all of its terms made this kernel nine tenths of the solver's time.)
+constexpr int UINV_WARPS = 16;
+__global__ void __launch_bounds__(32 * UINV_WARPS) uinv_row_kernel(const double* __restrict__ U, double* __restrict__ V, int64_t K, int i) {
+  __shared__ double part[UINV_WARPS][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int64_t c = (int64_t)i + 1 + (int64_t)blockIdx.x * 32 + lane;
   const double* ui = U + (int64_t)i * K;
-  const double inv = 1.0 / ui[i];
-  if (c == i) { V[(int64_t)i * K + i] = inv; return; }
   double s = 0.0;
-  for (int64_t k = i + 1; k <= c; ++k) s += ui[k] * V[k * K + c];
-  V[(int64_t)i * K + c] = -s * inv;
+  if (c < K)
+    for (int64_t k = (int64_t)i + 1 + w; k <= c; k += UINV_WARPS) s += ui[k] * V[k * K + c];
+  part[w][lane] = s;
+  __syncthreads();
+  const double inv = 1.0 / ui[i];
+  if (w == 0 && c < K) {
+    double t = 0.0;
+#pragma unroll
+    for (int q = 0; q < UINV_WARPS; ++q) t += part[q][lane];
+    V[(int64_t)i * K + c] = -t * inv;
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) V[(int64_t)i * K + i] = inv;
 }
 __global__ void zero_lower_kernel(double* __restrict__ V, int64_t K) {       // strictly lower part of V := 0
   for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < K * K; idx += (int64_t)gridDim.x * blockDim.x)
@@ -410,7 +422,7 @@ static cudaError_t gptq_run(const void* W, int64_t N, int64_t K, const void* Xc,
   }
   zero_lower_kernel<<<1184, 256, 0, st>>>(V, K); GQ_CHECK();
   for (int i = (int)K - 1; i >= 0; --i) {                 // V = U^-1, last row first
-    uinv_row_kernel<<<(unsigned)((K - i + 255) / 256), 256, 0, st>>>(A, V, K, i); GQ_CHECK();
+    uinv_row_kernel<<<(unsigned)((K - i - 1 + 31) / 32 > 0 ? (K - i - 1 + 31) / 32 : 1), 32 * UINV_WARPS, 0, st>>>(A, V, K, i); GQ_CHECK();
   }
   __nv_bfloat16* Tb = reinterpret_cast<__nv_bfloat16*>(T);
   for (int i = 0; i < C; ++i) {
